@@ -1,0 +1,193 @@
+/* rk.h -- C ABI of the B200 (sm_100a) MLA-Online step of RedKnot-MLA.
+ *
+ * One online layer (Algorithm 2 "Relocate, recompute, and merge one online layer"):
+ *   for every document segment i:  q_i = R(-delta_i) q;  SelectiveMLA(q_i, C_i, A)
+ *   SegmentedLSEMerge over segments;  z_online = W_{a,G} O_G + W_{a,L} O_{L,A};
+ *   z = RestoreAndReplace(z_off, z_online, A);  y = W_b z.
+ *
+ * Conventions
+ *  - Every function returns an rk_status (0 = RK_OK) and never throws.  All argument errors
+ *    are found on the host before anything is enqueued.  rk_last_error() gives a message.
+ *  - "device" pointers are CUDA device memory owned by the caller; "host" pointers are
+ *    ordinary host memory that is copied during the call and not retained.
+ *  - bf16 tensors are passed as `const void*` holding 16-bit bfloat16 (the bits of
+ *    torch.bfloat16 / __nv_bfloat16); all tensors are dense row-major, innermost dimension
+ *    contiguous, base pointers 16-byte aligned.
+ *  - Rows are in PACKED order: document 0, 1, ..., then the query suffix -- the order of the
+ *    packed latent stream.  Packed row r of segment i sits at request position
+ *    pos[r] = seg_delta[i] + (r - seg_off[i]).  Row t sees key k iff pos[k] <= pos[t].
+ *  - `stream` is a cudaStream_t (0 = default stream).  Calls enqueue work and return; the
+ *    only blocking calls are rk_create / rk_request_create / rk_poll_status / *_destroy and
+ *    rk_layer_host.
+ *  - The library allocates device memory only inside rk_create and rk_request_create (small
+ *    tables) and frees it in the matching destroy.  kv, weights and z_off are never written.
+ *  - No kernel traps: a device-side wait that expires records RK_ERR_TIMEOUT in a status
+ *    word, the kernel drains and returns; rk_poll_status() reads (and clears) that word.
+ *  - There is no fallback: rk_create fails with RK_ERR_UNSUPPORTED on a device that is not
+ *    compute capability 10.x.
+ */
+#ifndef RK_H_
+#define RK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum rk_status {
+  RK_OK = 0,
+  RK_ERR_NULL = 1,        /* a required pointer is NULL */
+  RK_ERR_PROFILE = 2,     /* head/group geometry inconsistent */
+  RK_ERR_LAYOUT = 3,      /* segment table invalid */
+  RK_ERR_ROWS = 4,        /* protected-row list invalid */
+  RK_ERR_ALIGN = 5,       /* pointer or stride not 16-byte aligned */
+  RK_ERR_WORKSPACE = 6,   /* workspace too small */
+  RK_ERR_UNSUPPORTED = 7, /* dims / device not supported */
+  RK_ERR_CUDA = 8,        /* a CUDA call failed */
+  RK_ERR_TIMEOUT = 9      /* a bounded device-side wait expired */
+} rk_status;
+
+/* Head partition and projection geometry (Eq. partition; Section "DeepSeek-V4 Flash and Pro
+ * profiles": one Global head per native group of eight).  Supported: group_size 8,
+ * d_latent 512, d_rope 64, d_v 128; o_rank and d_model multiples of 128. */
+typedef struct rk_profile {
+  int32_t n_heads;              /* H */
+  int32_t n_groups;             /* G = H / group_size */
+  int32_t group_size;           /* 8 */
+  int32_t d_latent;             /* 512: width of the shared latent c (also the value width) */
+  int32_t d_rope;               /* 64 */
+  int32_t d_v;                  /* 128: per-head width after W_uv */
+  int32_t o_rank;               /* r_o: rows of each group's block of W_a */
+  int32_t d_model;              /* rows of W_b */
+  float sm_scale;               /* softmax scale applied to q.k */
+  float rope_base;              /* theta_j = rope_base^(-2j/d_rope), interleaved pairs */
+  const int32_t* global_heads;  /* host [n_groups]: absolute index of each group's Global head,
+                                   global_heads[g] / group_size == g */
+} rk_profile;
+
+/* Segment geometry of one request (Section "Online position restoration and segmented
+ * merge"): document i was built at positions 0..n_i-1 and appears at request offset
+ * seg_delta[i].  Request-position intervals must not overlap; gaps are legal. */
+typedef struct rk_layout {
+  int32_t n_segs;
+  const int64_t* seg_off;          /* host [n_segs+1], packed-row prefix sums, seg_off[0] = 0 */
+  const int64_t* seg_delta;        /* host [n_segs], >= 0 */
+  const uint8_t* seg_has_artifact; /* host [n_segs]; 0 = no offline artifact (all its rows must be protected) */
+} rk_layout;
+
+typedef struct rk_request_info {
+  int64_t n_rows;        /* T */
+  int64_t n_prot;        /* A */
+  int64_t n_off_rows;    /* rows the z_off tensor must have (end of the last segment with artifact) */
+  int64_t pairs_global;  /* visible (row,key) pairs summed over rows: T(T+1)/2 for gap-free layouts */
+  int64_t pairs_local;   /* visible pairs summed over protected rows */
+  int32_t n_tiles_global;
+  int32_t n_tiles_local;
+} rk_request_info;
+
+typedef struct rk_ctx rk_ctx;
+typedef struct rk_request rk_request;
+
+const char* rk_version(void);
+const char* rk_status_string(rk_status s);
+
+/* Creates a context on the CURRENT CUDA device.  Copies the profile (including global_heads). */
+rk_status rk_create(const rk_profile* profile, rk_ctx** out);
+rk_status rk_destroy(rk_ctx* ctx);
+/* Message of the last failing call on this context (valid until the next call). */
+const char* rk_last_error(const rk_ctx* ctx);
+/* Synchronises `stream`, returns the device status word (RK_OK or RK_ERR_TIMEOUT) and clears it. */
+rk_status rk_poll_status(rk_ctx* ctx, void* stream);
+/* Per-wait time limit of device-side waits, in milliseconds (default 2000). */
+rk_status rk_set_wait_limit_ms(rk_ctx* ctx, int32_t ms);
+
+/* Request geometry object: validates the layout and the protected-row list (Eq. protected;
+ * the list is data here), builds row positions, per-segment relocation tables
+ * cos/sin(delta_i * theta_j) in double precision, the inverse row map and the tile work
+ * lists, and uploads them.  prot_rows: host [n_prot], strictly ascending packed rows; must
+ * contain every row of every segment without artifact.  Reusable across layers and calls. */
+rk_status rk_request_create(rk_ctx* ctx, const rk_layout* layout, const int32_t* prot_rows, int64_t n_prot,
+                            rk_request** out);
+rk_status rk_request_destroy(rk_request* req);
+/* The same validation as rk_request_create, on the host only (no device, no context): returns the
+ * status rk_request_create would return for this layout / row list and writes a message into msg
+ * (may be NULL). */
+rk_status rk_check_request(const rk_layout* layout, const int32_t* prot_rows, int64_t n_prot, char* msg,
+                           size_t msg_len);
+rk_status rk_request_get_info(const rk_request* req, rk_request_info* out);
+/* Bytes of device scratch that rk_group_sliced_proj needs (per-head o = W_uv O_lat in bf16). */
+rk_status rk_workspace_bytes(const rk_request* req, size_t* out);
+
+/* (1) Query-side RoPE relocation, standalone form (Algorithm 2: q_i <- R(-delta_i) q; Eq. rope).
+ * q_rope: device bf16, rope sub-vectors (64 wide) of n_rows x n_heads queries already rotated at
+ * their request positions; element (r, h, e) at q_rope[r*row_stride + h*head_stride + e]
+ * (strides in elements, multiples of 8).  out: device bf16 [seg_end-seg_begin][n_rows][n_heads][64],
+ * out[i] = R(-seg_delta[seg_begin+i]) q.  The same rotation is fused into rk_mla_online_attn. */
+rk_status rk_relocate_q(rk_ctx* ctx, const rk_request* req, const void* q_rope, int64_t n_rows, int32_t n_heads,
+                        int64_t row_stride, int64_t head_stride, int32_t seg_begin, int32_t seg_end, void* out,
+                        void* stream);
+
+/* (2) Absorbed-MLA attention over the packed latent (Algorithm 2: SelectiveMLA for every
+ * segment + running SegmentedLSEMerge inside the kernel; relocation fused into the Q load).
+ *   kv   device bf16 [T][576] = [c (512) | k_rope at the document's canonical position (64)]
+ *   q_g  device bf16 [T][G][576]  queries of the Global heads (group order), request position
+ *   q_l  device bf16 [A][L][576]  queries of the Local heads (ascending head index) on the
+ *        protected rows in list order
+ *   O_g  device bf16 [T][G][512], lse_g device fp32 [T][G]   (natural-log LSE of scaled scores)
+ *   O_l  device bf16 [A][L][512], lse_l device fp32 [A][L]
+ * Either pass may be skipped by passing NULL for its q, O and lse. */
+rk_status rk_mla_online_attn(rk_ctx* ctx, const rk_request* req, const void* kv, const void* q_g, const void* q_l,
+                             void* O_g, float* lse_g, void* O_l, float* lse_l, void* stream);
+
+/* (3) Stable segmented log-sum-exp merge, standalone form (Algorithm 2: SegmentedLSEMerge):
+ * lse = log sum_j exp(lse_j), O = sum_j exp(lse_j - lse) O_j over n_parts partial results.
+ *   O_part   device [n_parts][n_rows][n_heads][512], bf16 (part_dtype 0) or fp32 (part_dtype 1)
+ *   lse_part device fp32 [n_parts][n_rows][n_heads]; -inf marks an empty part (its O is ignored)
+ *   O device bf16 [n_rows][n_heads][512], lse device fp32 [n_rows][n_heads]
+ * All parts empty gives O = 0, lse = -inf. */
+rk_status rk_segmented_merge(rk_ctx* ctx, int32_t n_parts, int64_t n_rows, int32_t n_heads, const void* O_part,
+                             int32_t part_dtype, const float* lse_part, void* O, float* lse, void* stream);
+
+/* (4) Group-aligned sliced first output projection (Eq. offonline; Algorithm 2: z_online):
+ * per head o = W_uv[h] O_lat (512 -> 128), then the head's 128-column slice of its group's W_a:
+ *   z_on_g[t][g] = W_a[g][:, 128 j_g : 128 j_g + 128] o[t][global head of g]         (all T rows)
+ *   z_on_l[a][g] = sum over the 7 Local heads j of group g of W_a[g][:, 128 j : ..] o[a][8g+j]
+ *   W_uv device bf16 [H][128][512];  W_a device bf16 [G][r_o][1024]
+ *   z_on_g device bf16 [T][G*r_o];   z_on_l device bf16 [A][G*r_o]
+ * workspace: device scratch of at least rk_workspace_bytes().  Either half may be skipped by
+ * passing NULL for its O and z. */
+rk_status rk_group_sliced_proj(rk_ctx* ctx, const rk_request* req, const void* O_g, const void* O_l,
+                               const void* W_uv, const void* W_a, void* z_on_g, void* z_on_l, void* workspace,
+                               size_t workspace_bytes, void* stream);
+
+/* (5) Add the offline MLA-Off artifact and run the shared second projection (Algorithm 2:
+ * RestoreAndReplace, then W_b z; "replaced, never double counted"):
+ *   z[t] = z_on_g[t] + (t in A ? z_on_l[slot(t)] : z_off[t]);  y = W_b z.
+ *   z_off device bf16 [n_off_rows][G*r_o] (packed rows; rows in A are never read)
+ *   W_b   device bf16 [d_model][G*r_o], may be NULL to stop at z
+ *   z     device bf16 [T][G*r_o] (required);  y device bf16 [T][d_model] (required iff W_b) */
+rk_status rk_combine_offline(rk_ctx* ctx, const rk_request* req, const void* z_on_g, const void* z_on_l,
+                             const void* z_off, const void* W_b, void* z, void* y, void* stream);
+
+/* Device buffers that rk_layer_host stages through; all owned by the caller. */
+typedef struct rk_layer_buffers {
+  void *kv, *q_g, *q_l, *z_off;            /* device copies of the per-request inputs */
+  void *O_g, *O_l, *z_on_g, *z_on_l, *z, *y;
+  float *lse_g, *lse_l;
+  void* workspace;
+  size_t workspace_bytes;
+} rk_layer_buffers;
+
+/* One whole layer from HOST inputs: copies kv, q_g, q_l, z_off host->device (pinned host
+ * memory recommended), runs (2), (4), (5) on `stream`, copies y device->host and synchronises
+ * the stream.  Weights stay resident on the device. */
+rk_status rk_layer_host(rk_ctx* ctx, const rk_request* req, const void* kv_host, const void* q_g_host,
+                        const void* q_l_host, const void* z_off_host, const void* W_uv, const void* W_a,
+                        const void* W_b, const rk_layer_buffers* dev, void* y_host, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RK_H_ */

@@ -1,0 +1,630 @@
+// Host side of the C ABI: argument validation, request geometry (row positions, relocation
+// tables, inverse row map, tile work lists), TMA tensor maps and kernel launches.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/rk.h"
+#include "rk_internal.h"
+
+using namespace rk;
+
+// ------------------------------------------------------------------------------------------
+// objects
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct rk_ctx {
+  rk_profile prof;
+  std::vector<int32_t> global_heads, local_heads;
+  int device = 0;
+  int sm_count = 0;
+  int n_pairs = 0;
+  DeviceStatus* d_status = nullptr;
+  GemmBatch* d_batches = nullptr;  // [uv_g: G][uv_l: L][wa_g: G][wa_l: G][wb: 1]
+  int off_uv_g = 0, off_uv_l = 0, off_wa_g = 0, off_wa_l = 0, off_wb = 0;
+  unsigned long long wait_ns = 2000ull * 1000 * 1000;
+  PFN_encodeTiled encode = nullptr;
+  mutable std::string err;
+};
+
+struct rk_request {
+  rk_ctx* ctx = nullptr;
+  int64_t T = 0, A = 0, n_off_rows = 0;
+  int32_t S = 0;
+  int64_t pairs_global = 0, pairs_local = 0;
+  int32_t n_tiles_g = 0, n_tiles_l = 0;
+  // device tables
+  int32_t* d_row_pos = nullptr;
+  int32_t* d_prot_rows = nullptr;
+  int32_t* d_inv_map = nullptr;
+  int32_t* d_seg_off = nullptr;
+  int32_t* d_seg_delta = nullptr;
+  float2* d_seg_cs = nullptr;
+  AttnWorkItem* d_work_g = nullptr;
+  AttnWorkItem* d_work_l = nullptr;
+};
+
+namespace {
+
+rk_status fail(const rk_ctx* ctx, rk_status s, const char* fmt, ...) {
+  if (ctx) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    ctx->err = buf;
+  }
+  return s;
+}
+
+rk_status cuda_fail(const rk_ctx* ctx, cudaError_t e, const char* what) {
+  cudaGetLastError();
+  return fail(ctx, RK_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <class T>
+cudaError_t upload(T** dst, const std::vector<T>& v) {
+  *dst = nullptr;
+  size_t bytes = std::max<size_t>(v.size(), 1) * sizeof(T);
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(dst), bytes);
+  if (e != cudaSuccess) return e;
+  if (!v.empty()) e = cudaMemcpy(*dst, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice);
+  return e;
+}
+
+// 2-D bf16 row-major tensor map with 128-byte swizzle; box = box_cols x box_rows.
+rk_status make_tmap(const rk_ctx* ctx, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                    uint64_t row_stride_elems, uint32_t box_cols, uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {row_stride_elems * 2};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return fail(ctx, RK_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) rows=%llu cols=%llu stride=%llu", (int)r,
+                (unsigned long long)rows, (unsigned long long)cols, (unsigned long long)row_stride_elems);
+  return RK_OK;
+}
+
+void build_work(const std::vector<int32_t>& tok_pos, int hpt, const std::vector<int32_t>& seg_n,
+                const std::vector<int32_t>& seg_delta, int n_pairs, std::vector<AttnWorkItem>* out) {
+  const int64_t n_flat = (int64_t)tok_pos.size() * hpt;
+  const int64_t n_tiles = (n_flat + kAttnRowsPerPair - 1) / kAttnRowsPerPair;
+  std::vector<std::pair<int64_t, AttnWorkItem>> items((size_t)n_tiles);
+  for (int64_t t = 0; t < n_tiles; ++t) {
+    const int64_t r0 = t * kAttnRowsPerPair, r1 = std::min<int64_t>(n_flat, r0 + kAttnRowsPerPair);
+    const int64_t tok0 = r0 / hpt, tok1 = (r1 - 1) / hpt;
+    int32_t maxpos = 0;
+    for (int64_t k = tok0; k <= tok1; ++k) maxpos = std::max(maxpos, tok_pos[(size_t)k]);
+    int64_t cost = 0;
+    for (size_t i = 0; i < seg_n.size(); ++i) {
+      int64_t kmax = std::min<int64_t>(seg_n[i], (int64_t)maxpos - seg_delta[i] + 1);
+      if (kmax > 0) cost += (kmax + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
+    }
+    items[(size_t)t] = {cost, AttnWorkItem{(int32_t)t, maxpos}};
+  }
+  std::stable_sort(items.begin(), items.end(),
+                   [](const auto& a, const auto& b) { return a.first > b.first; });
+  // longest first; every other round of n_pairs tiles is reversed so that the static
+  // round-robin assignment (pair p takes entries p, p + n_pairs, ...) stays balanced
+  out->resize((size_t)n_tiles);
+  for (int64_t base = 0, round = 0; base < n_tiles; base += n_pairs, ++round) {
+    const int64_t cnt = std::min<int64_t>(n_pairs, n_tiles - base);
+    for (int64_t k = 0; k < cnt; ++k) {
+      const int64_t src = (round & 1) ? (base + cnt - 1 - k) : (base + k);
+      (*out)[(size_t)(base + k)] = items[(size_t)src].second;
+    }
+  }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+extern "C" {
+
+const char* rk_version(void) { return "rk-mla-online 0.1 (sm_100a)"; }
+
+const char* rk_status_string(rk_status s) {
+  switch (s) {
+    case RK_OK: return "RK_OK";
+    case RK_ERR_NULL: return "RK_ERR_NULL";
+    case RK_ERR_PROFILE: return "RK_ERR_PROFILE";
+    case RK_ERR_LAYOUT: return "RK_ERR_LAYOUT";
+    case RK_ERR_ROWS: return "RK_ERR_ROWS";
+    case RK_ERR_ALIGN: return "RK_ERR_ALIGN";
+    case RK_ERR_WORKSPACE: return "RK_ERR_WORKSPACE";
+    case RK_ERR_UNSUPPORTED: return "RK_ERR_UNSUPPORTED";
+    case RK_ERR_CUDA: return "RK_ERR_CUDA";
+    case RK_ERR_TIMEOUT: return "RK_ERR_TIMEOUT";
+  }
+  return "RK_ERR_?";
+}
+
+const char* rk_last_error(const rk_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
+  if (!prof || !out) return RK_ERR_NULL;
+  *out = nullptr;
+  if (!prof->global_heads) return RK_ERR_NULL;
+  if (prof->group_size != kGroup || prof->d_latent != kDLatent || prof->d_rope != kDRope || prof->d_v != kDV)
+    return RK_ERR_UNSUPPORTED;
+  if (prof->n_groups <= 0 || prof->n_heads != prof->n_groups * prof->group_size) return RK_ERR_PROFILE;
+  if (prof->o_rank <= 0 || prof->o_rank % 128 != 0 || prof->d_model <= 0 || prof->d_model % 128 != 0)
+    return RK_ERR_UNSUPPORTED;
+  if (!(prof->sm_scale > 0.f) || !(prof->rope_base > 1.f)) return RK_ERR_PROFILE;
+  for (int g = 0; g < prof->n_groups; ++g) {
+    const int h = prof->global_heads[g];
+    if (h < 0 || h >= prof->n_heads || h / prof->group_size != g) return RK_ERR_PROFILE;
+  }
+  rk_ctx* ctx = new (std::nothrow) rk_ctx();
+  if (!ctx) return RK_ERR_CUDA;
+  ctx->prof = *prof;
+  ctx->global_heads.assign(prof->global_heads, prof->global_heads + prof->n_groups);
+  ctx->prof.global_heads = ctx->global_heads.data();
+  for (int h = 0; h < prof->n_heads; ++h)
+    if (ctx->global_heads[h / kGroup] != h) ctx->local_heads.push_back(h);
+
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  cudaDeviceProp dp;
+  if (e == cudaSuccess) e = cudaGetDeviceProperties(&dp, ctx->device);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    delete ctx;
+    return RK_ERR_CUDA;
+  }
+  if (dp.major != 10) {  // tcgen05 / TMEM path only; there is no fallback
+    delete ctx;
+    return RK_ERR_UNSUPPORTED;
+  }
+  ctx->sm_count = dp.multiProcessorCount;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+    cudaGetLastError();
+    delete ctx;
+    return RK_ERR_CUDA;
+  }
+  ctx->encode = reinterpret_cast<PFN_encodeTiled>(fn);
+  e = attention_setup();
+  if (e == cudaSuccess) e = gemm_setup();
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->d_status), sizeof(DeviceStatus));
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(DeviceStatus));
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    delete ctx;
+    return RK_ERR_CUDA;
+  }
+  ctx->n_pairs = attention_max_pairs(ctx->sm_count);
+
+  // GEMM batch tables (depend only on the head partition)
+  const int G = prof->n_groups, L = (int)ctx->local_heads.size(), ro = prof->o_rank;
+  const int32_t kNoSkip = 1 << 30;
+  std::vector<GemmBatch> b;
+  ctx->off_uv_g = (int)b.size();
+  for (int g = 0; g < G; ++g) b.push_back(GemmBatch{g * kDLatent, ctx->global_heads[g] * kDV, 0, kNoSkip, g * kDV, {0, 0, 0}});
+  ctx->off_uv_l = (int)b.size();
+  for (int l = 0; l < L; ++l) b.push_back(GemmBatch{l * kDLatent, ctx->local_heads[l] * kDV, 0, kNoSkip, l * kDV, {0, 0, 0}});
+  ctx->off_wa_g = (int)b.size();
+  for (int g = 0; g < G; ++g) {
+    const int j = ctx->global_heads[g] % kGroup;
+    b.push_back(GemmBatch{g * kDV, g * ro, j * kDV, kNoSkip, g * ro, {0, 0, 0}});
+  }
+  ctx->off_wa_l = (int)b.size();
+  for (int g = 0; g < G; ++g) {
+    const int j = ctx->global_heads[g] % kGroup;
+    b.push_back(GemmBatch{g * (kGroup - 1) * kDV, g * ro, 0, j * kDV, g * ro, {0, 0, 0}});
+  }
+  ctx->off_wb = (int)b.size();
+  b.push_back(GemmBatch{0, 0, 0, kNoSkip, 0, {0, 0, 0}});
+  e = upload(&ctx->d_batches, b);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(ctx->d_status);
+    if (ctx->d_batches) cudaFree(ctx->d_batches);
+    delete ctx;
+    return RK_ERR_CUDA;
+  }
+  *out = ctx;
+  return RK_OK;
+}
+
+rk_status rk_destroy(rk_ctx* ctx) {
+  if (!ctx) return RK_ERR_NULL;
+  cudaFree(ctx->d_status);
+  cudaFree(ctx->d_batches);
+  delete ctx;
+  return RK_OK;
+}
+
+rk_status rk_set_wait_limit_ms(rk_ctx* ctx, int32_t ms) {
+  if (!ctx) return RK_ERR_NULL;
+  if (ms <= 0) return fail(ctx, RK_ERR_PROFILE, "wait limit must be positive");
+  ctx->wait_ns = (unsigned long long)ms * 1000ull * 1000ull;
+  return RK_OK;
+}
+
+rk_status rk_poll_status(rk_ctx* ctx, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  cudaError_t e = cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamSynchronize");
+  DeviceStatus h;
+  e = cudaMemcpy(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "status readback");
+  if (h.code != 0) {
+    cudaMemset(ctx->d_status, 0, sizeof(DeviceStatus));
+    return fail(ctx, RK_ERR_TIMEOUT, "device wait expired: tag %d, block %d, aux %d", h.where, h.block, h.aux);
+  }
+  return RK_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Pure host check of a layout and a protected-row list (no device needed).  msg may be NULL.
+rk_status rk_check_request(const rk_layout* lay, const int32_t* prot_rows, int64_t n_prot, char* msg,
+                           size_t msg_len) {
+  auto bad = [&](rk_status s, const char* fmt, long long a, long long b) {
+    if (msg && msg_len) snprintf(msg, msg_len, fmt, a, b);
+    return s;
+  };
+  if (!lay || !lay->seg_off || !lay->seg_delta || !lay->seg_has_artifact || (n_prot > 0 && !prot_rows))
+    return bad(RK_ERR_NULL, "null argument", 0, 0);
+  const int S = lay->n_segs;
+  if (S <= 0) return bad(RK_ERR_LAYOUT, "n_segs must be positive", 0, 0);
+  if (lay->seg_off[0] != 0) return bad(RK_ERR_LAYOUT, "seg_off[0] must be 0", 0, 0);
+  for (int i = 0; i < S; ++i) {
+    if (lay->seg_off[i + 1] <= lay->seg_off[i])
+      return bad(RK_ERR_LAYOUT, "segment %lld is empty or seg_off is not increasing", i, 0);
+    if (lay->seg_delta[i] < 0) return bad(RK_ERR_LAYOUT, "segment %lld has a negative request offset", i, 0);
+    if (lay->seg_delta[i] + (lay->seg_off[i + 1] - lay->seg_off[i]) >= (int64_t)1 << 30)
+      return bad(RK_ERR_LAYOUT, "segment %lld reaches request position 2^30 or beyond", i, 0);
+  }
+  const int64_t T = lay->seg_off[S];
+  if (T >= ((int64_t)1 << 30)) return bad(RK_ERR_LAYOUT, "too many rows", 0, 0);
+  {  // request-position intervals must not overlap
+    std::vector<std::pair<int64_t, int64_t>> iv;
+    for (int i = 0; i < S; ++i)
+      iv.push_back({lay->seg_delta[i], lay->seg_delta[i] + lay->seg_off[i + 1] - lay->seg_off[i]});
+    std::sort(iv.begin(), iv.end());
+    for (int i = 1; i < S; ++i)
+      if (iv[i].first < iv[i - 1].second)
+        return bad(RK_ERR_LAYOUT, "request-position intervals overlap at position %lld", iv[i].first, 0);
+  }
+  if (n_prot < 0 || n_prot > T) return bad(RK_ERR_ROWS, "n_prot out of range", 0, 0);
+  std::vector<uint8_t> is_prot((size_t)T, 0);
+  for (int64_t a = 0; a < n_prot; ++a) {
+    const int64_t r = prot_rows[a];
+    if (r < 0 || r >= T) return bad(RK_ERR_ROWS, "protected row %lld out of range", r, 0);
+    if (a > 0 && prot_rows[a] <= prot_rows[a - 1])
+      return bad(RK_ERR_ROWS, "protected rows must be strictly ascending (entry %lld)", a, 0);
+    is_prot[(size_t)r] = 1;
+  }
+  for (int i = 0; i < S; ++i)
+    if (!lay->seg_has_artifact[i])
+      for (int64_t r = lay->seg_off[i]; r < lay->seg_off[i + 1]; ++r)
+        if (!is_prot[(size_t)r])
+          return bad(RK_ERR_ROWS, "row %lld of segment %lld has no artifact and is not protected", r, i);
+  return RK_OK;
+}
+
+rk_status rk_request_create(rk_ctx* ctx, const rk_layout* lay, const int32_t* prot_rows, int64_t n_prot,
+                            rk_request** out) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!out) return fail(ctx, RK_ERR_NULL, "null argument");
+  *out = nullptr;
+  {
+    char msg[256] = {0};
+    rk_status s = rk_check_request(lay, prot_rows, n_prot, msg, sizeof(msg));
+    if (s != RK_OK) return fail(ctx, s, "%s", msg);
+  }
+  const int S = lay->n_segs;
+  const int64_t T = lay->seg_off[S];
+  std::vector<int32_t> inv((size_t)T, -1);
+  for (int64_t a = 0; a < n_prot; ++a) inv[(size_t)prot_rows[a]] = (int32_t)a;
+  int64_t n_off_rows = 0;
+  for (int i = 0; i < S; ++i)
+    if (lay->seg_has_artifact[i]) n_off_rows = lay->seg_off[i + 1];
+
+  rk_request* rq = new (std::nothrow) rk_request();
+  if (!rq) return fail(ctx, RK_ERR_CUDA, "out of host memory");
+  rq->ctx = ctx;
+  rq->T = T;
+  rq->A = n_prot;
+  rq->S = S;
+  rq->n_off_rows = n_off_rows;
+
+  std::vector<int32_t> seg_off32((size_t)S + 1), seg_delta32((size_t)S), seg_n((size_t)S), row_pos((size_t)T);
+  for (int i = 0; i <= S; ++i) seg_off32[(size_t)i] = (int32_t)lay->seg_off[i];
+  for (int i = 0; i < S; ++i) {
+    seg_delta32[(size_t)i] = (int32_t)lay->seg_delta[i];
+    seg_n[(size_t)i] = seg_off32[(size_t)i + 1] - seg_off32[(size_t)i];
+    for (int64_t r = lay->seg_off[i]; r < lay->seg_off[i + 1]; ++r)
+      row_pos[(size_t)r] = (int32_t)(lay->seg_delta[i] + (r - lay->seg_off[i]));
+  }
+  // relocation tables: angle delta_i * theta_j evaluated in double, theta_j = base^(-2j/d_rope)
+  std::vector<float2> cs((size_t)S * 32);
+  for (int i = 0; i < S; ++i)
+    for (int j = 0; j < 32; ++j) {
+      const double theta = std::pow((double)ctx->prof.rope_base, -2.0 * j / (double)kDRope);
+      const double ang = (double)lay->seg_delta[i] * theta;
+      cs[(size_t)i * 32 + j] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+    }
+  // visible-pair counts (for flop accounting): keys with pos <= row pos
+  auto visible = [&](int64_t pos) {
+    int64_t v = 0;
+    for (int i = 0; i < S; ++i) v += std::max<int64_t>(0, std::min<int64_t>(seg_n[(size_t)i], pos - seg_delta32[(size_t)i] + 1));
+    return v;
+  };
+  for (int64_t r = 0; r < T; ++r) rq->pairs_global += visible(row_pos[(size_t)r]);
+  std::vector<int32_t> prot((size_t)n_prot), prot_pos((size_t)n_prot);
+  for (int64_t a = 0; a < n_prot; ++a) {
+    prot[(size_t)a] = prot_rows[a];
+    prot_pos[(size_t)a] = row_pos[(size_t)prot_rows[a]];
+    rq->pairs_local += visible(prot_pos[(size_t)a]);
+  }
+  std::vector<AttnWorkItem> work_g, work_l;
+  build_work(row_pos, ctx->prof.n_groups, seg_n, seg_delta32, ctx->n_pairs, &work_g);
+  build_work(prot_pos, (int)ctx->local_heads.size(), seg_n, seg_delta32, ctx->n_pairs, &work_l);
+  rq->n_tiles_g = (int32_t)work_g.size();
+  rq->n_tiles_l = (int32_t)work_l.size();
+
+  cudaError_t e = upload(&rq->d_row_pos, row_pos);
+  if (e == cudaSuccess) e = upload(&rq->d_prot_rows, prot);
+  if (e == cudaSuccess) e = upload(&rq->d_inv_map, inv);
+  if (e == cudaSuccess) e = upload(&rq->d_seg_off, seg_off32);
+  if (e == cudaSuccess) e = upload(&rq->d_seg_delta, seg_delta32);
+  if (e == cudaSuccess) e = upload(&rq->d_seg_cs, cs);
+  if (e == cudaSuccess) e = upload(&rq->d_work_g, work_g);
+  if (e == cudaSuccess) e = upload(&rq->d_work_l, work_l);
+  if (e != cudaSuccess) {
+    rk_request_destroy(rq);
+    return cuda_fail(ctx, e, "request table upload");
+  }
+  *out = rq;
+  return RK_OK;
+}
+
+rk_status rk_request_destroy(rk_request* rq) {
+  if (!rq) return RK_ERR_NULL;
+  cudaFree(rq->d_row_pos);
+  cudaFree(rq->d_prot_rows);
+  cudaFree(rq->d_inv_map);
+  cudaFree(rq->d_seg_off);
+  cudaFree(rq->d_seg_delta);
+  cudaFree(rq->d_seg_cs);
+  cudaFree(rq->d_work_g);
+  cudaFree(rq->d_work_l);
+  delete rq;
+  return RK_OK;
+}
+
+rk_status rk_request_get_info(const rk_request* rq, rk_request_info* out) {
+  if (!rq || !out) return RK_ERR_NULL;
+  out->n_rows = rq->T;
+  out->n_prot = rq->A;
+  out->n_off_rows = rq->n_off_rows;
+  out->pairs_global = rq->pairs_global;
+  out->pairs_local = rq->pairs_local;
+  out->n_tiles_global = rq->n_tiles_g;
+  out->n_tiles_local = rq->n_tiles_l;
+  return RK_OK;
+}
+
+static size_t proj_ws_bytes(const rk_request* rq) {
+  const rk_ctx* c = rq->ctx;
+  const size_t og = ((size_t)rq->T * c->prof.n_groups * kDV * 2 + 255) & ~(size_t)255;
+  const size_t ol = ((size_t)rq->A * c->local_heads.size() * kDV * 2 + 255) & ~(size_t)255;
+  return og + ol;
+}
+
+rk_status rk_workspace_bytes(const rk_request* rq, size_t* out) {
+  if (!rq || !out) return RK_ERR_NULL;
+  *out = proj_ws_bytes(rq);
+  return RK_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+rk_status rk_relocate_q(rk_ctx* ctx, const rk_request* rq, const void* q_rope, int64_t n_rows, int32_t n_heads,
+                        int64_t row_stride, int64_t head_stride, int32_t seg_begin, int32_t seg_end, void* out,
+                        void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!rq || !q_rope || !out) return fail(ctx, RK_ERR_NULL, "null argument");
+  if (rq->ctx != ctx) return fail(ctx, RK_ERR_LAYOUT, "request belongs to another context");
+  if (n_rows < 0 || n_heads <= 0) return fail(ctx, RK_ERR_LAYOUT, "bad row/head count");
+  if (seg_begin < 0 || seg_end > rq->S || seg_begin > seg_end) return fail(ctx, RK_ERR_LAYOUT, "segment range out of bounds");
+  if (!aligned16(q_rope) || !aligned16(out) || row_stride % 8 != 0 || head_stride % 8 != 0)
+    return fail(ctx, RK_ERR_ALIGN, "q_rope/out must be 16-byte aligned and strides multiples of 8 elements");
+  if (head_stride < kDRope || row_stride < head_stride) return fail(ctx, RK_ERR_LAYOUT, "strides too small");
+  cudaError_t e = launch_relocate(q_rope, n_rows, n_heads, row_stride, head_stride, rq->d_seg_cs, seg_begin, seg_end,
+                                  out, ctx->sm_count, reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "relocate launch");
+}
+
+static rk_status attn_pass(rk_ctx* ctx, const rk_request* rq, const void* kv, const void* q, int64_t n_tok, int hpt,
+                           const int32_t* rowmap, const AttnWorkItem* work, int n_tiles, void* O, float* lse,
+                           cudaStream_t stream) {
+  if (n_tiles == 0) return RK_OK;
+  AttnParams p;
+  memset(&p, 0, sizeof(p));
+  const int64_t n_flat = n_tok * hpt;
+  rk_status s = make_tmap(ctx, &p.tm_q, q, (uint64_t)n_flat, kDQK, kDQK, 64, kAttnRowsPerCta);
+  if (s != RK_OK) return s;
+  s = make_tmap(ctx, &p.tm_kv, kv, (uint64_t)rq->T, kDQK, kDQK, 64, 128);
+  if (s != RK_OK) return s;
+  p.row_pos = rq->d_row_pos;
+  p.rowmap = rowmap;
+  p.seg_off = rq->d_seg_off;
+  p.seg_delta = rq->d_seg_delta;
+  p.seg_cs = rq->d_seg_cs;
+  p.work = work;
+  p.O = O;
+  p.lse = lse;
+  p.status = ctx->d_status;
+  p.wait_ns = ctx->wait_ns;
+  p.n_segs = rq->S;
+  p.n_tiles = n_tiles;
+  p.n_flat = (int32_t)n_flat;
+  p.hpt = hpt;
+  const int n_pairs = std::min(ctx->n_pairs, n_tiles);
+  p.n_pairs = n_pairs;
+  p.scale_log2 = ctx->prof.sm_scale * 1.44269504088896340736f;
+  cudaError_t e = launch_attention(p, n_pairs, stream);
+  return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "attention launch");
+}
+
+rk_status rk_mla_online_attn(rk_ctx* ctx, const rk_request* rq, const void* kv, const void* q_g, const void* q_l,
+                             void* O_g, float* lse_g, void* O_l, float* lse_l, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!rq || !kv) return fail(ctx, RK_ERR_NULL, "null argument");
+  if (rq->ctx != ctx) return fail(ctx, RK_ERR_LAYOUT, "request belongs to another context");
+  const bool do_g = q_g || O_g || lse_g, do_l = q_l || O_l || lse_l;
+  if (do_g && !(q_g && O_g && lse_g)) return fail(ctx, RK_ERR_NULL, "Global pass needs q_g, O_g and lse_g");
+  if (do_l && !(q_l && O_l && lse_l)) return fail(ctx, RK_ERR_NULL, "Local pass needs q_l, O_l and lse_l");
+  if (!aligned16(kv) || !aligned16(q_g) || !aligned16(q_l) || !aligned16(O_g) || !aligned16(O_l))
+    return fail(ctx, RK_ERR_ALIGN, "tensor base pointers must be 16-byte aligned");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  rk_status s = RK_OK;
+  if (do_g)
+    s = attn_pass(ctx, rq, kv, q_g, rq->T, ctx->prof.n_groups, nullptr, rq->d_work_g, rq->n_tiles_g, O_g, lse_g, st);
+  if (s == RK_OK && do_l && rq->A > 0)
+    s = attn_pass(ctx, rq, kv, q_l, rq->A, (int)ctx->local_heads.size(), rq->d_prot_rows, rq->d_work_l, rq->n_tiles_l,
+                  O_l, lse_l, st);
+  return s;
+}
+
+rk_status rk_segmented_merge(rk_ctx* ctx, int32_t n_parts, int64_t n_rows, int32_t n_heads, const void* O_part,
+                             int32_t part_dtype, const float* lse_part, void* O, float* lse, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!O_part || !lse_part || !O || !lse) return fail(ctx, RK_ERR_NULL, "null argument");
+  if (n_parts <= 0 || n_parts > 4096 || n_rows < 0 || n_heads <= 0) return fail(ctx, RK_ERR_LAYOUT, "bad part/row/head count");
+  if (part_dtype != 0 && part_dtype != 1) return fail(ctx, RK_ERR_UNSUPPORTED, "part_dtype must be 0 (bf16) or 1 (fp32)");
+  if (!aligned16(O_part) || !aligned16(O)) return fail(ctx, RK_ERR_ALIGN, "O_part/O must be 16-byte aligned");
+  cudaError_t e = launch_merge(n_parts, n_rows * n_heads, O_part, part_dtype, lse_part, O, lse, ctx->sm_count,
+                               reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "merge launch");
+}
+
+static rk_status run_gemm(rk_ctx* ctx, const void* A, int64_t a_rows, int64_t a_cols, const void* B, int64_t b_rows,
+                          int64_t b_cols, void* C, int64_t ldc, int M, int N, int K, int batch_off, int n_batches,
+                          cudaStream_t st) {
+  if (M == 0) return RK_OK;
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  const int bn = (N % 256 == 0) ? 256 : 128;
+  rk_status s = make_tmap(ctx, &p.tm_a, A, (uint64_t)a_rows, (uint64_t)a_cols, (uint64_t)a_cols, 64, 128);
+  if (s != RK_OK) return s;
+  s = make_tmap(ctx, &p.tm_b, B, (uint64_t)b_rows, (uint64_t)b_cols, (uint64_t)b_cols, 64, (uint32_t)bn);
+  if (s != RK_OK) return s;
+  p.C = C;
+  p.batches = ctx->d_batches + batch_off;
+  p.status = ctx->d_status;
+  p.wait_ns = ctx->wait_ns;
+  p.ldc = ldc;
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  p.n_batches = n_batches;
+  cudaError_t e = launch_gemm(p, bn, st);
+  return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "gemm launch");
+}
+
+rk_status rk_group_sliced_proj(rk_ctx* ctx, const rk_request* rq, const void* O_g, const void* O_l, const void* W_uv,
+                               const void* W_a, void* z_on_g, void* z_on_l, void* workspace, size_t workspace_bytes,
+                               void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!rq || !W_uv || !W_a || !workspace) return fail(ctx, RK_ERR_NULL, "null argument");
+  if (rq->ctx != ctx) return fail(ctx, RK_ERR_LAYOUT, "request belongs to another context");
+  const bool do_g = O_g || z_on_g, do_l = O_l || z_on_l;
+  if (do_g && !(O_g && z_on_g)) return fail(ctx, RK_ERR_NULL, "Global half needs O_g and z_on_g");
+  if (do_l && !(O_l && z_on_l)) return fail(ctx, RK_ERR_NULL, "Local half needs O_l and z_on_l");
+  if (!aligned16(O_g) || !aligned16(O_l) || !aligned16(W_uv) || !aligned16(W_a) || !aligned16(z_on_g) ||
+      !aligned16(z_on_l) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return fail(ctx, RK_ERR_ALIGN, "tensors must be 16-byte aligned and the workspace 256-byte aligned");
+  if (workspace_bytes < proj_ws_bytes(rq)) return fail(ctx, RK_ERR_WORKSPACE, "workspace too small: need %zu bytes", proj_ws_bytes(rq));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int G = ctx->prof.n_groups, H = ctx->prof.n_heads, L = H - G, ro = ctx->prof.o_rank;
+  const int64_t T = rq->T, A = rq->A;
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  void* o_g = ws;
+  void* o_l = ws + (((size_t)T * G * kDV * 2 + 255) & ~(size_t)255);
+  rk_status s = RK_OK;
+  if (do_g) {
+    s = run_gemm(ctx, O_g, T, (int64_t)G * kDLatent, W_uv, (int64_t)H * kDV, kDLatent, o_g, (int64_t)G * kDV, (int)T, kDV,
+                 kDLatent, ctx->off_uv_g, G, st);
+    if (s == RK_OK)
+      s = run_gemm(ctx, o_g, T, (int64_t)G * kDV, W_a, (int64_t)G * ro, kGroup * kDV, z_on_g, (int64_t)G * ro, (int)T, ro,
+                   kDV, ctx->off_wa_g, G, st);
+  }
+  if (s == RK_OK && do_l && A > 0) {
+    s = run_gemm(ctx, O_l, A, (int64_t)L * kDLatent, W_uv, (int64_t)H * kDV, kDLatent, o_l, (int64_t)L * kDV, (int)A, kDV,
+                 kDLatent, ctx->off_uv_l, L, st);
+    if (s == RK_OK)
+      s = run_gemm(ctx, o_l, A, (int64_t)L * kDV, W_a, (int64_t)G * ro, kGroup * kDV, z_on_l, (int64_t)G * ro, (int)A, ro,
+                   (kGroup - 1) * kDV, ctx->off_wa_l, G, st);
+  }
+  return s;
+}
+
+rk_status rk_combine_offline(rk_ctx* ctx, const rk_request* rq, const void* z_on_g, const void* z_on_l,
+                             const void* z_off, const void* W_b, void* z, void* y, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!rq || !z_on_g || !z) return fail(ctx, RK_ERR_NULL, "null argument");
+  if (rq->ctx != ctx) return fail(ctx, RK_ERR_LAYOUT, "request belongs to another context");
+  if (rq->A > 0 && !z_on_l) return fail(ctx, RK_ERR_NULL, "z_on_l is required when rows are protected");
+  if (rq->A < rq->T && !z_off) return fail(ctx, RK_ERR_NULL, "z_off is required when some rows are not protected");
+  if (W_b && !y) return fail(ctx, RK_ERR_NULL, "y is required when W_b is given");
+  if (!aligned16(z_on_g) || !aligned16(z_on_l) || !aligned16(z_off) || !aligned16(W_b) || !aligned16(z) || !aligned16(y))
+    return fail(ctx, RK_ERR_ALIGN, "tensor base pointers must be 16-byte aligned");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int64_t width = (int64_t)ctx->prof.n_groups * ctx->prof.o_rank;
+  cudaError_t e = launch_combine(z_on_g, z_on_l, z_off, rq->d_inv_map, rq->T, width, z, ctx->sm_count, st);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "combine launch");
+  if (!W_b) return RK_OK;
+  return run_gemm(ctx, z, rq->T, width, W_b, ctx->prof.d_model, width, y, ctx->prof.d_model, (int)rq->T,
+                  ctx->prof.d_model, (int)width, ctx->off_wb, 1, st);
+}
+
+rk_status rk_layer_host(rk_ctx* ctx, const rk_request* rq, const void* kv_host, const void* q_g_host,
+                        const void* q_l_host, const void* z_off_host, const void* W_uv, const void* W_a,
+                        const void* W_b, const rk_layer_buffers* dev, void* y_host, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!rq || !kv_host || !q_g_host || !W_uv || !W_a || !W_b || !dev || !y_host) return fail(ctx, RK_ERR_NULL, "null argument");
+  if (rq->ctx != ctx) return fail(ctx, RK_ERR_LAYOUT, "request belongs to another context");
+  if (rq->A > 0 && !q_l_host) return fail(ctx, RK_ERR_NULL, "q_l_host is required");
+  if (rq->A < rq->T && !z_off_host) return fail(ctx, RK_ERR_NULL, "z_off_host is required");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int G = ctx->prof.n_groups, L = ctx->prof.n_heads - G;
+  const size_t width = (size_t)G * ctx->prof.o_rank;
+  cudaError_t e = cudaMemcpyAsync(dev->kv, kv_host, (size_t)rq->T * kDQK * 2, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dev->q_g, q_g_host, (size_t)rq->T * G * kDQK * 2, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && rq->A > 0)
+    e = cudaMemcpyAsync(dev->q_l, q_l_host, (size_t)rq->A * L * kDQK * 2, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && rq->n_off_rows > 0 && z_off_host)
+    e = cudaMemcpyAsync(dev->z_off, z_off_host, (size_t)rq->n_off_rows * width * 2, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "host to device copy");
+  rk_status s = rk_mla_online_attn(ctx, rq, dev->kv, dev->q_g, rq->A > 0 ? dev->q_l : nullptr, dev->O_g, dev->lse_g,
+                                   rq->A > 0 ? dev->O_l : nullptr, rq->A > 0 ? dev->lse_l : nullptr, stream);
+  if (s == RK_OK)
+    s = rk_group_sliced_proj(ctx, rq, dev->O_g, rq->A > 0 ? dev->O_l : nullptr, W_uv, W_a, dev->z_on_g,
+                             rq->A > 0 ? dev->z_on_l : nullptr, dev->workspace, dev->workspace_bytes, stream);
+  if (s == RK_OK) s = rk_combine_offline(ctx, rq, dev->z_on_g, dev->z_on_l, dev->z_off, W_b, dev->z, dev->y, stream);
+  if (s != RK_OK) return s;
+  e = cudaMemcpyAsync(y_host, dev->y, (size_t)rq->T * ctx->prof.d_model * 2, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "device to host copy");
+}
+
+}  // extern "C"

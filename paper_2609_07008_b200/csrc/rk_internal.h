@@ -1,0 +1,86 @@
+// Internal declarations shared by the host layer and the kernel launchers (not part of the ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rk_ptx.cuh"
+
+namespace rk {
+
+constexpr int kDLatent = 512;
+constexpr int kDRope = 64;
+constexpr int kDQK = 576;
+constexpr int kDV = 128;
+constexpr int kGroup = 8;
+
+// ---- attention -----------------------------------------------------------------------
+constexpr int kAttnRowsPerCta = 64;    // query rows (token x head pairs) per CTA
+constexpr int kAttnRowsPerPair = 128;  // per CTA pair (one UMMA M=128 across two SMs)
+constexpr int kAttnKeysPerTile = 256;  // keys per UMMA N
+
+struct AttnWorkItem {
+  int32_t tile;    // flattened-row tile index (128 rows each)
+  int32_t maxpos;  // largest request position among the tile's rows
+};
+
+struct AttnParams {
+  CUtensorMap tm_q;   // [n_flat][576] bf16, box 64 cols x 64 rows, 128B swizzle
+  CUtensorMap tm_kv;  // [T][576] bf16, box 64 cols x 128 rows, 128B swizzle
+  const int32_t* row_pos;    // [T] request position of each packed row
+  const int32_t* rowmap;     // [n_tok] token slot -> packed row, or nullptr (identity)
+  const int32_t* seg_off;    // [S+1]
+  const int32_t* seg_delta;  // [S]
+  const float2* seg_cs;      // [S][32] (cos, sin)(delta_i * theta_j)
+  const AttnWorkItem* work;  // [n_tiles] cost-descending
+  void* O;                   // bf16 [n_flat][512]
+  float* lse;                // [n_flat]
+  DeviceStatus* status;
+  unsigned long long wait_ns;
+  int32_t n_segs;
+  int32_t n_tiles;
+  int32_t n_flat;  // tokens * heads_per_token
+  int32_t hpt;     // heads per token in this pass (G or L)
+  int32_t n_pairs;
+  float scale_log2;  // sm_scale * log2(e)
+};
+
+cudaError_t launch_attention(const AttnParams& p, int n_pairs, cudaStream_t stream);
+cudaError_t attention_setup();  // sets the dynamic shared memory attribute once
+int attention_max_pairs(int sm_count);
+
+// ---- batched GEMM  C[M,N] = A[M,K] * B[N,K]^T  (bf16 in, fp32 accumulate, bf16 out) ----------
+struct GemmBatch {
+  int32_t a_col0;   // column offset of this batch's A block
+  int32_t b_row0;   // row offset of this batch's B block
+  int32_t b_col0;   // column offset of this batch's B block
+  int32_t b_skip;   // K index at which a 128-column hole starts in B (or a huge value)
+  int32_t c_col0;   // column offset of this batch's C block
+  int32_t pad[3];
+};
+
+struct GemmParams {
+  CUtensorMap tm_a;  // [M rows][a_cols] box 64 x 128
+  CUtensorMap tm_b;  // [b_rows][b_cols] box 64 x BN
+  void* C;
+  const GemmBatch* batches;
+  DeviceStatus* status;
+  unsigned long long wait_ns;
+  int64_t ldc;  // elements
+  int32_t M, N, K;
+  int32_t n_batches;
+};
+
+cudaError_t launch_gemm(const GemmParams& p, int bn, cudaStream_t stream);
+cudaError_t gemm_setup();
+
+// ---- streaming kernels -----------------------------------------------------------------------
+cudaError_t launch_relocate(const void* q_rope, int64_t n_rows, int32_t n_heads, int64_t row_stride,
+                            int64_t head_stride, const float2* seg_cs, int32_t seg_begin, int32_t seg_end,
+                            void* out, int sm_count, cudaStream_t stream);
+cudaError_t launch_merge(int32_t n_parts, int64_t n_rh, const void* O_part, int32_t part_dtype,
+                         const float* lse_part, void* O, float* lse, int sm_count, cudaStream_t stream);
+cudaError_t launch_combine(const void* z_on_g, const void* z_on_l, const void* z_off, const int32_t* inv_map,
+                           int64_t T, int64_t width, void* z, int sm_count, cudaStream_t stream);
+
+}  // namespace rk

@@ -1,0 +1,196 @@
+// HBM-bound steps of the MLA-Online layer: standalone query relocation (Algorithm 2,
+// q_i = R(-delta_i) q), standalone segmented log-sum-exp merge (SegmentedLSEMerge) and
+// restore-and-replace (z = z_on_g + (row in A ? z_on_l : z_off)).  16-byte vector accesses,
+// consecutive threads on consecutive addresses, grids sized in multiples of the SM count.
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "rk_internal.h"
+
+namespace rk {
+namespace {
+
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    __nv_bfloat162 x = *reinterpret_cast<const __nv_bfloat162*>(&w[e]);
+    f[2 * e] = __bfloat162float(x.x);
+    f[2 * e + 1] = __bfloat162float(x.y);
+  }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+  return make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+}
+
+// One thread per 16-byte chunk (4 rotation pairs) of one (row, head); the input is read once
+// and one rotated copy is written per segment frame.
+__global__ void __launch_bounds__(256) rk_relocate_kernel(const __nv_bfloat16* __restrict__ q, int64_t n_rows,
+                                                          int32_t n_heads, int64_t row_stride, int64_t head_stride,
+                                                          const float2* __restrict__ seg_cs, int32_t seg_begin,
+                                                          int32_t n_frames, __nv_bfloat16* __restrict__ out) {
+  const int64_t n_items = n_rows * n_heads * 8;
+  const int64_t frame_elems = n_rows * n_heads * 64;
+  for (int64_t it = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; it < n_items;
+       it += (int64_t)gridDim.x * blockDim.x) {
+    const int c = (int)(it & 7);
+    const int64_t rh = it >> 3;
+    const int64_t r = rh / n_heads;
+    const int h = (int)(rh - r * n_heads);
+    const uint4 v = *reinterpret_cast<const uint4*>(q + r * row_stride + h * head_stride + c * 8);
+    float x[8];
+    unpack8(v, x);
+    __nv_bfloat16* dst = out + it * 8;
+#pragma unroll 4
+    for (int i = 0; i < n_frames; ++i) {
+      const float4* cs = reinterpret_cast<const float4*>(seg_cs + (size_t)(seg_begin + i) * 32 + 4 * c);
+      const float4 t01 = __ldg(cs), t23 = __ldg(cs + 1);
+      float y[8];
+      // R(-delta): (x0, x1) -> (x0 cos + x1 sin, x1 cos - x0 sin)
+      y[0] = x[0] * t01.x + x[1] * t01.y;  y[1] = x[1] * t01.x - x[0] * t01.y;
+      y[2] = x[2] * t01.z + x[3] * t01.w;  y[3] = x[3] * t01.z - x[2] * t01.w;
+      y[4] = x[4] * t23.x + x[5] * t23.y;  y[5] = x[5] * t23.x - x[4] * t23.y;
+      y[6] = x[6] * t23.z + x[7] * t23.w;  y[7] = x[7] * t23.z - x[6] * t23.w;
+      __stcs(reinterpret_cast<uint4*>(dst + (int64_t)i * frame_elems), pack8(y));
+    }
+  }
+}
+
+// One warp per (row, head): weights from the per-part LSE (max-subtracted), then the weighted
+// sum of the 512-wide partial outputs; lane l owns dims [8l, 8l+8) and [256+8l, 256+8l+8).
+template <bool kF32>
+__global__ void __launch_bounds__(256) rk_merge_kernel(int32_t n_parts, int64_t n_rh, const void* __restrict__ O_part,
+                                                       const float* __restrict__ lse_part,
+                                                       __nv_bfloat16* __restrict__ O, float* __restrict__ lse) {
+  extern __shared__ float wsm[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float* w = wsm + (size_t)warp * n_parts;
+  const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  for (int64_t rh = (int64_t)blockIdx.x * (blockDim.x >> 5) + warp; rh < n_rh; rh += n_warps) {
+    float mx = -INFINITY;
+    for (int j = lane; j < n_parts; j += 32) {
+      const float l = __ldg(lse_part + (int64_t)j * n_rh + rh);
+      w[j] = l;
+      mx = fmaxf(mx, l);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    const float m_safe = (mx == -INFINITY) ? 0.f : mx;
+    float tot = 0.f;
+    __syncwarp();
+    for (int j = lane; j < n_parts; j += 32) {
+      const float e = __expf(w[j] - m_safe);  // exp(-inf) = 0 for empty parts
+      w[j] = e;
+      tot += e;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+    __syncwarp();
+    const float inv = tot > 0.f ? 1.f / tot : 0.f;
+    float acc[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+    for (int j = 0; j < n_parts; ++j) {
+      const float wj = w[j] * inv;
+      if (wj > 0.f) {
+        if (kF32) {
+          const float* src = reinterpret_cast<const float*>(O_part) + ((int64_t)j * n_rh + rh) * 512;
+#pragma unroll
+          for (int hlf = 0; hlf < 2; ++hlf) {
+            const float4 a = __ldcs(reinterpret_cast<const float4*>(src + 256 * hlf + 8 * lane));
+            const float4 b = __ldcs(reinterpret_cast<const float4*>(src + 256 * hlf + 8 * lane + 4));
+            acc[8 * hlf + 0] += wj * a.x; acc[8 * hlf + 1] += wj * a.y; acc[8 * hlf + 2] += wj * a.z; acc[8 * hlf + 3] += wj * a.w;
+            acc[8 * hlf + 4] += wj * b.x; acc[8 * hlf + 5] += wj * b.y; acc[8 * hlf + 6] += wj * b.z; acc[8 * hlf + 7] += wj * b.w;
+          }
+        } else {
+          const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(O_part) + ((int64_t)j * n_rh + rh) * 512;
+#pragma unroll
+          for (int hlf = 0; hlf < 2; ++hlf) {
+            const uint4 v = __ldcs(reinterpret_cast<const uint4*>(src + 256 * hlf + 8 * lane));
+            float f[8];
+            unpack8(v, f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[8 * hlf + e] += wj * f[e];
+          }
+        }
+      }
+    }
+    __nv_bfloat16* dst = O + rh * 512;
+    *reinterpret_cast<uint4*>(dst + 8 * lane) = pack8(acc);
+    *reinterpret_cast<uint4*>(dst + 256 + 8 * lane) = pack8(acc + 8);
+    if (lane == 0) lse[rh] = tot > 0.f ? m_safe + logf(tot) : -INFINITY;
+    __syncwarp();
+  }
+}
+
+// z = z_on_g + (protected ? z_on_l[slot] : z_off[row]): a per-row select, never an add of both.
+__global__ void __launch_bounds__(256) rk_combine_kernel(const __nv_bfloat16* __restrict__ z_on_g,
+                                                         const __nv_bfloat16* __restrict__ z_on_l,
+                                                         const __nv_bfloat16* __restrict__ z_off,
+                                                         const int32_t* __restrict__ inv_map, int64_t T, int64_t width,
+                                                         __nv_bfloat16* __restrict__ z) {
+  const int64_t cpr = width >> 3;  // 16-byte chunks per row
+  const int64_t n_items = T * cpr;
+  for (int64_t it = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; it < n_items;
+       it += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t t = it / cpr;
+    const int64_t c = it - t * cpr;
+    const int32_t slot = __ldg(inv_map + t);
+    const uint4 a = __ldcs(reinterpret_cast<const uint4*>(z_on_g + t * width) + c);
+    const uint4 b = slot >= 0 ? __ldcs(reinterpret_cast<const uint4*>(z_on_l + (int64_t)slot * width) + c)
+                              : __ldcs(reinterpret_cast<const uint4*>(z_off + t * width) + c);
+    float fa[8], fb[8];
+    unpack8(a, fa);
+    unpack8(b, fb);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) fa[e] += fb[e];
+    *(reinterpret_cast<uint4*>(z + t * width) + c) = pack8(fa);
+  }
+}
+
+inline int grid_for(int64_t n_threads_needed, int sm_count, int per_sm) {
+  int64_t blocks = (n_threads_needed + 255) / 256;
+  int64_t cap = (int64_t)sm_count * per_sm;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return (int)blocks;
+}
+
+}  // namespace
+
+cudaError_t launch_relocate(const void* q_rope, int64_t n_rows, int32_t n_heads, int64_t row_stride,
+                            int64_t head_stride, const float2* seg_cs, int32_t seg_begin, int32_t seg_end, void* out,
+                            int sm_count, cudaStream_t stream) {
+  const int64_t items = n_rows * n_heads * 8;
+  if (items == 0 || seg_end <= seg_begin) return cudaSuccess;
+  rk_relocate_kernel<<<grid_for(items, sm_count, 8), 256, 0, stream>>>(
+      reinterpret_cast<const __nv_bfloat16*>(q_rope), n_rows, n_heads, row_stride, head_stride, seg_cs, seg_begin,
+      seg_end - seg_begin, reinterpret_cast<__nv_bfloat16*>(out));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_merge(int32_t n_parts, int64_t n_rh, const void* O_part, int32_t part_dtype, const float* lse_part,
+                         void* O, float* lse, int sm_count, cudaStream_t stream) {
+  if (n_rh == 0) return cudaSuccess;
+  const size_t smem = (size_t)8 * n_parts * sizeof(float);
+  const int grid = grid_for(n_rh * 32, sm_count, 8);
+  if (part_dtype == 1)
+    rk_merge_kernel<true><<<grid, 256, smem, stream>>>(n_parts, n_rh, O_part, lse_part,
+                                                        reinterpret_cast<__nv_bfloat16*>(O), lse);
+  else
+    rk_merge_kernel<false><<<grid, 256, smem, stream>>>(n_parts, n_rh, O_part, lse_part,
+                                                         reinterpret_cast<__nv_bfloat16*>(O), lse);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const void* z_on_g, const void* z_on_l, const void* z_off, const int32_t* inv_map, int64_t T,
+                           int64_t width, void* z, int sm_count, cudaStream_t stream) {
+  const int64_t items = T * (width >> 3);
+  if (items == 0) return cudaSuccess;
+  rk_combine_kernel<<<grid_for(items, sm_count, 8), 256, 0, stream>>>(
+      reinterpret_cast<const __nv_bfloat16*>(z_on_g), reinterpret_cast<const __nv_bfloat16*>(z_on_l),
+      reinterpret_cast<const __nv_bfloat16*>(z_off), inv_map, T, width, reinterpret_cast<__nv_bfloat16*>(z));
+  return cudaGetLastError();
+}
+
+}  // namespace rk

@@ -1,0 +1,223 @@
+"""GPU parity: every C-ABI call against the float64 checker on identical seeded inputs
+(bf16 storage, fp32 accumulate).  Tolerances: max-abs <= 1e-2 and relative L2 <= 5e-3 per
+tensor; one-rounding steps (relocation) are held to one bf16 ulp; selections are bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_07008_b200 import synth
+from tests.helpers import assert_close, f64, max_abs, oracle_online, rel_l2, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rk():
+    from paper_2609_07008_b200 import binding
+    return binding
+
+
+def make(rk, w):
+    ctx = rk.Context.from_profile(w.profile)
+    req = ctx.rk_request_create(w.layout.seg_off, w.layout.seg_delta, w.layout.seg_has_artifact, w.prot_rows)
+    return ctx, req
+
+
+def small_ragged(regime="sharp", seed=5):
+    return synth.make_custom([300, 77, 513], 50, n_heads=16, n_groups=2, o_rank=256, d_model=512, pct_bp=700,
+                             seed=seed, regime=regime)
+
+
+# -- (1) relocation ---------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("name", ["tiny", "ragged"])
+def test_relocate_q(rk, name):
+    w = synth.make_workload("tiny") if name == "tiny" else small_ragged()
+    ctx, req = make(rk, w)
+    to_device(w)
+    S = w.layout.n_segs
+    view = w.q_g[:, :, 512:]                       # strided view of the rope sub-vectors
+    out = ctx.rk_relocate_q(req, view, 0, S)
+    ctx.rk_poll_status()
+    x = f64(view)
+    for i in range(S):
+        want = oracle.relocate_query(x, float(w.layout.seg_delta[i]), w.profile.rope_base)
+        got = f64(out[i])
+        err = np.abs(got - want)
+        assert (err <= 2.0 ** -8 * np.abs(want) + 1e-6 * np.abs(x).max()).all(), f"segment {i}: {err.max()}"
+    # a sub-range of segments lands in the right frames
+    out2 = ctx.rk_relocate_q(req, view, 1, S)
+    assert torch.equal(out2, out[1:])
+
+
+# -- (3) standalone merge ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("P", [1, 3, 65])
+def test_segmented_merge(rk, dtype, P):
+    w = synth.make_workload("tiny")
+    ctx, _ = make(rk, w)
+    g = torch.Generator().manual_seed(P)
+    n_rows, n_heads = 37, 5
+    O_part = torch.randn((P, n_rows, n_heads, 512), generator=g).to(dtype)
+    lse_part = torch.randn((P, n_rows, n_heads), generator=g) * 3
+    if P > 1:
+        lse_part[torch.rand((P, n_rows, n_heads), generator=g) < 0.3] = -float("inf")
+        lse_part[:, 0, 0] = -float("inf")                      # a (row, head) whose parts are all empty
+        O_part[1, 1, 1] = float("nan")                         # ignored: its part is empty
+        lse_part[1, 1, 1] = -float("inf")
+    O, lse = ctx.rk_segmented_merge(O_part.cuda(), lse_part.cuda())
+    ctx.rk_poll_status()
+    want_O, want_lse = oracle.segmented_merge(f64(O_part), f64(lse_part))
+    got_lse = f64(lse)
+    fin = np.isfinite(want_lse)
+    assert np.array_equal(np.isneginf(got_lse), np.isneginf(want_lse))
+    assert max_abs(got_lse[fin], want_lse[fin]) <= 1e-3
+    assert_close(f64(O), want_O, "merged O")
+    if P == 1:
+        assert torch.equal(O.cpu(), O_part[0].to(torch.bfloat16))    # one part is the identity
+
+
+# -- (2) attention -----------------------------------------------------------------------------------
+
+def check_attention(rk, w, rows=None):
+    ctx, req = make(rk, w)
+    T = w.layout.n_rows
+    rows = np.arange(T) if rows is None else rows
+    exp = oracle_online(w, rows)
+    to_device(w)
+    O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
+    ctx.rk_poll_status()
+    r1 = assert_close(f64(O_g)[rows], exp["O_g"], "O_g")
+    assert max_abs(f64(lse_g)[rows], exp["lse_g"]) <= 1e-3
+    inv = oracle.inverse_row_map(w.prot_rows, T)
+    slots = inv[rows][inv[rows] >= 0]
+    r2 = assert_close(f64(O_l)[slots], exp["O_l"], "O_l")
+    assert max_abs(f64(lse_l)[slots], exp["lse_l"]) <= 1e-3
+    return r1, r2
+
+
+@pytest.mark.parametrize("regime", ["mandated", "sharp"])
+def test_attention_tiny(rk, regime):
+    check_attention(rk, synth.make_workload("tiny", regime=regime))
+
+
+@pytest.mark.parametrize("seed", [5, 6])
+def test_attention_ragged(rk, seed):
+    check_attention(rk, small_ragged(seed=seed))
+
+
+def test_attention_single_pass_and_shift(rk):
+    """Each pass can run alone; adding a constant to every request offset (and re-rotating q)
+    leaves the outputs unchanged within rounding."""
+    w = small_ragged(seed=7)
+    ctx, req = make(rk, w)
+    to_device(w)
+    O_g, lse_g, _, _ = ctx.rk_mla_online_attn(req, w.kv, w.q_g, None)
+    _, _, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, None, w.q_l)
+    O_g2, lse_g2, O_l2, lse_l2 = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
+    ctx.rk_poll_status()
+    assert torch.equal(O_g, O_g2) and torch.equal(O_l, O_l2) and torch.equal(lse_g, lse_g2)
+
+
+# -- (4) sliced projection ------------------------------------------------------------------------------
+
+def test_group_sliced_proj(rk):
+    w = small_ragged(seed=8)
+    ctx, req = make(rk, w)
+    p = w.profile
+    T, A = w.layout.n_rows, len(w.prot_rows)
+    g = torch.Generator().manual_seed(1)
+    O_g = (torch.randn((T, p.n_groups, 512), generator=g) * 0.5).to(torch.bfloat16)
+    O_l = (torch.randn((A, p.n_local, 512), generator=g) * 0.5).to(torch.bfloat16)
+    to_device(w)
+    z_on_g, z_on_l = ctx.rk_group_sliced_proj(req, O_g.cuda(), O_l.cuda(), w.w_uv, w.w_a)
+    ctx.rk_poll_status()
+    wuv, wa = f64(w.w_uv), f64(w.w_a)
+    cg = oracle.head_contributions(f64(O_g), p.global_heads, wuv, wa)
+    want_g = cg.reshape(T, -1)                                  # one Global head per group, group order
+    cl = oracle.head_contributions(f64(O_l), p.local_heads, wuv, wa)
+    want_l = np.zeros((A, p.n_groups, p.o_rank))
+    for a, h in enumerate(p.local_heads):
+        want_l[:, h // 8] += cl[:, a]
+    assert_close(f64(z_on_g), want_g, "z_on_g")
+    assert_close(f64(z_on_l), want_l.reshape(A, -1), "z_on_l")
+    # wrong-slice detector: zero one Local head's slice of W_a -> exactly that head's contribution goes
+    h = int(p.local_heads[4])
+    wa2 = w.w_a.clone()
+    wa2[h // 8, :, 128 * (h % 8):128 * (h % 8 + 1)] = 0
+    _, z2 = ctx.rk_group_sliced_proj(req, None, O_l.cuda(), w.w_uv, wa2)
+    ctx.rk_poll_status()
+    want2 = want_l.copy()
+    want2[:, h // 8] -= cl[:, 4]
+    assert_close(f64(z2), want2.reshape(A, -1), "z_on_l with one slice zeroed")
+
+
+# -- (5) combine + W_b -----------------------------------------------------------------------------------
+
+def test_combine_offline(rk):
+    w = small_ragged(seed=9)
+    ctx, req = make(rk, w)
+    p = w.profile
+    T, A = w.layout.n_rows, len(w.prot_rows)
+    width = p.n_groups * p.o_rank
+    g = torch.Generator().manual_seed(2)
+    z_on_g = (torch.randn((T, width), generator=g) * 0.3).to(torch.bfloat16)
+    z_on_l = (torch.randn((A, width), generator=g) * 0.3).to(torch.bfloat16)
+    z_off = (torch.randn((w.layout.n_doc_rows, width), generator=g) * 0.3).to(torch.bfloat16)
+    to_device(w)
+    z, y = ctx.rk_combine_offline(req, z_on_g.cuda(), z_on_l.cuda(), z_off.cuda(), w.w_b)
+    ctx.rk_poll_status()
+    inv = oracle.inverse_row_map(w.prot_rows, T)
+    want_z = f64(z_on_g).copy()
+    for t in range(T):
+        want_z[t] += f64(z_on_l[inv[t]]) if inv[t] >= 0 else f64(z_off[t])
+    assert_close(f64(z), want_z, "z")
+    assert_close(f64(y), f64(z) @ f64(w.w_b).T, "y from the library's own z")
+    assert_close(f64(y), want_z @ f64(w.w_b).T, "y")
+    # replaced, never double counted: poisoning z_off on protected rows changes nothing
+    z_poison = z_off.clone()
+    doc_prot = torch.as_tensor(w.prot_rows[w.prot_rows < w.layout.n_doc_rows].astype(np.int64))
+    z_poison[doc_prot] = float("nan")
+    zp = z_poison.cuda()
+    before = zp.clone()
+    z2, y2 = ctx.rk_combine_offline(req, z_on_g.cuda(), z_on_l.cuda(), zp, w.w_b)
+    ctx.rk_poll_status()
+    assert torch.equal(z2, z) and torch.equal(y2, y)
+    assert torch.equal(zp.view(torch.int16), before.view(torch.int16))     # the artifact is never written
+
+
+# -- end to end ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("regime", ["mandated", "sharp"])
+def test_end_to_end_tiny_honest_artifact(rk, regime):
+    w = synth.make_workload("tiny", regime=regime, with_q_all=True)
+    p, lay = w.profile, w.layout
+    # honest MLA-Off artifact from the checker (each document alone at position zero)
+    z_off = np.zeros((lay.n_doc_rows, p.n_groups * p.o_rank))
+    q_all = f64(w.q_all)
+    for i in range(lay.n_segs):
+        if lay.seg_has_artifact[i]:
+            lo, hi = int(lay.seg_off[i]), int(lay.seg_off[i + 1])
+            z_off[lo:hi] = oracle.mla_off_artifact(i, q_all[lo:hi][:, p.local_heads], f64(w.kv), lay.seg_off,
+                                                   lay.seg_delta, p.local_heads, f64(w.w_uv), f64(w.w_a), p.sm_scale,
+                                                   p.rope_base, p.d_latent)
+    w.z_off = torch.from_numpy(z_off).to(torch.bfloat16)
+    rows = np.arange(lay.n_rows)
+    exp = oracle_online(w, rows)
+    ctx, req = make(rk, w)
+    to_device(w)
+    O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
+    z_on_g, z_on_l = ctx.rk_group_sliced_proj(req, O_g, O_l, w.w_uv, w.w_a)
+    z, y = ctx.rk_combine_offline(req, z_on_g, z_on_l, w.z_off, w.w_b)
+    ctx.rk_poll_status()
+    assert_close(f64(z), exp["z"], "z")
+    assert_close(f64(y), exp["y"], "y")
+    # the same through the host-buffer entry point
+    bufs = ctx.alloc_layer_buffers(req, "cuda")
+    pin = lambda t: t.cpu().pin_memory()
+    y_h = torch.empty((lay.n_rows, p.d_model), dtype=torch.bfloat16).pin_memory()
+    ctx.rk_layer_host(req, pin(w.kv), pin(w.q_g), pin(w.q_l), pin(w.z_off), w.w_uv, w.w_a, w.w_b, bufs, y_h)
+    ctx.rk_poll_status()
+    assert torch.equal(y_h, y.cpu())
