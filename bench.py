@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the MLA-Online layer (RedKnot-MLA, Algorithm 2) on B200.
+
+One step = one pass of the whole hot path over one synthetic request:
+rk_mla_online_attn (relocation fused, segments merged in-kernel) -> rk_group_sliced_proj ->
+rk_combine_offline (restore-and-replace + shared W_b).  Metric: prefill tokens/s per layer.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs its own independent request of
+the same shape (the path has no exchange step: weak scaling, no collective in the data path);
+the value is the total over ranks divided by the slowest rank's device time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_07008_b200 import synth  # noqa: E402
+
+FLOP_PER_PAIR = 2 * 576 + 2 * 512     # QK^T over 576 + PV over 512 per visible (row, key, head)
+L2_BYTES = 126 * 1024 * 1024
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_burst=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.stop_flag = index, [], False
+
+    def run(self):
+        while not self.stop_flag:
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                f = [x.strip() for x in out.strip().split(",")]
+                if len(f) >= 6:
+                    self.samples.append(f)
+            except Exception:
+                pass
+            time.sleep(0.2)
+
+    def summary(self):
+        if not self.samples:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["unavailable"])
+        mhz = sorted(int(s[0]) for s in self.samples if s[0].isdigit())
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
+        return dict(sm_mhz=mhz[len(mhz) // 2] if mhz else None, sm_max_mhz=int(self.samples[0][1]), reasons=reasons,
+                    samples=len(self.samples))
+
+
+def algorithmic_flops(profile, req):
+    """Work the method itself must do: Global heads x all rows + Local heads x protected rows."""
+    G, L, ro, dm = profile.n_groups, profile.n_local, profile.o_rank, profile.d_model
+    attn = FLOP_PER_PAIR * (G * req.pairs_global + L * req.pairs_local)
+    proj = 2 * req.T * G * (512 * 128 + 128 * ro) + 2 * req.A * (L * 512 * 128 + G * 7 * 128 * ro)
+    wb = 2 * req.T * G * ro * dm
+    return attn, proj, wb
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU checker timing (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample_run(w, rows):
+    """Runs the float64 checker on the packed rows `rows`; returns (seconds, visible pairs)."""
+    import oracle
+    from tests.helpers import f64
+    p, lay = w.profile, w.layout
+    rows = np.asarray(rows, dtype=np.int64)
+    inv = oracle.inverse_row_map(w.prot_rows, lay.n_rows)
+    ridx = torch.as_tensor(rows, device=w.q_g.device)
+    q_g_rows = f64(w.q_g[ridx])
+    ql = {int(r): f64(w.q_l[int(inv[r])]) for r in rows if inv[r] >= 0}
+    zo = {int(r): f64(w.z_off[int(r)]) for r in rows if inv[r] < 0}
+    kv, wuv, wa, wb = f64(w.kv), f64(w.w_uv), f64(w.w_a), f64(w.w_b)
+    pos = oracle.request_positions(lay.seg_off, lay.seg_delta)
+    srt = np.sort(pos)
+    vis = np.searchsorted(srt, pos[rows], side="right")
+    pairs = int(sum(v * (p.n_heads if inv[r] >= 0 else p.n_groups) for v, r in zip(vis, rows)))
+    t0 = time.perf_counter()
+    out = oracle.mla_online_rows(rows, q_g_rows, ql, kv, lay.seg_off, lay.seg_delta, w.prot_rows, p.global_heads,
+                                 p.local_heads, wuv, wa, wb, zo, p.sm_scale, p.rope_base, p.d_latent)
+    dt = time.perf_counter() - t0
+    return dt, pairs, out
+
+
+def pick_oracle_rows(w, pair_budget):
+    """Seeded sample of rows (half protected) whose visible-pair count stays within the budget."""
+    p, lay = w.profile, w.layout
+    cand = synth.sample_rows(lay, w.prot_rows, 64, w.seed)
+    import oracle
+    pos = oracle.request_positions(lay.seg_off, lay.seg_delta)
+    srt = np.sort(pos)
+    inv = oracle.inverse_row_map(w.prot_rows, lay.n_rows)
+    rng = np.random.default_rng(w.seed + 5)
+    cand = rng.permutation(cand)
+    rows, used = [], 0
+    for r in cand:
+        c = int(np.searchsorted(srt, pos[r], side="right")) * (p.n_heads if inv[r] >= 0 else p.n_groups)
+        if used + c > pair_budget and rows:
+            continue
+        rows.append(int(r))
+        used += c
+        if used >= pair_budget:
+            break
+    return np.sort(np.asarray(rows, dtype=np.int64))
+
+
+def total_pairs(profile, req):
+    return profile.n_groups * req.pairs_global + profile.n_local * req.pairs_local
+
+
+def run_reference(args, rank, world):
+    """--impl reference: the float64 CPU checker, as it stands, on the host cores; every step is
+    a bounded row sample of the same workload and tokens/s is extrapolated by visible pairs."""
+    if rank != 0:
+        return
+    name = args.config
+    prof, lay, prot = synth.make_geometry(name)
+    w = synth.make_tensors(name, prof, lay, prot, synth.CONFIGS[name]["seed"] * 1000, device="cpu")
+    import oracle
+    pos = oracle.request_positions(lay.seg_off, lay.seg_delta)
+    srt = np.sort(pos)
+    pg = int(np.searchsorted(srt, pos, side="right").sum())
+    pl = int(np.searchsorted(srt, pos[prot], side="right").sum())
+    all_pairs = prof.n_groups * pg + prof.n_local * pl
+    rows = pick_oracle_rows(w, args.oracle_pairs)
+    times, pairs = [], 0
+    for i in range(args.warmup + args.steps):
+        dt, pairs, _ = oracle_sample_run(w, rows)
+        if i >= args.warmup:
+            times.append(dt)
+    sec = float(np.mean(times))
+    tok_s = lay.n_rows / (sec * all_pairs / pairs)
+    cores = os.cpu_count()
+    line = dict(metric="mla_online_prefill_tokens_per_s_per_layer", value=tok_s, unit="tokens/s", n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=sec * 1e3 * all_pairs / pairs,
+                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                impl="reference", config=dict(workload=name, T=lay.n_rows, n_prot=len(prot)),
+                cpu_baseline=dict(value=tok_s, unit="tokens/s", cores=cores, kind="oracle",
+                                  sample=f"{len(rows)} seeded rows, {pairs} of {all_pairs} visible (row,key,head) "
+                                         f"pairs per step, extrapolated by pair count"),
+                e2e=dict(value=tok_s, unit="tokens/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="flash256k", choices=list(synth.CONFIGS))
+    ap.add_argument("--impl", default="rk", choices=["rk", "reference"])
+    ap.add_argument("--regime", default="mandated", choices=["mandated", "sharp"])
+    ap.add_argument("--oracle-pairs", type=int, default=150_000_000,
+                    help="visible-pair budget of the CPU checker sample (about 10-30 s of host work)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "rk" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch.distributed as dist
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2609_07008_b200 import binding as rk   # raises if librk.so is missing: no fallback
+
+    name = args.config
+    prof, lay, prot = synth.make_geometry(name)
+    # every rank gets its own request values (independent requests, same shape)
+    w = synth.make_tensors(name, prof, lay, prot, synth.CONFIGS[name]["seed"] * 1000 + rank, device=dev,
+                           regime=args.regime)
+    ctx = rk.Context.from_profile(prof)
+    req = ctx.rk_request_create(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, prot)
+    bufs = ctx.alloc_layer_buffers(req, dev)
+    fl_attn, fl_proj, fl_wb = algorithmic_flops(prof, req)
+    in_bytes = sum(t.numel() * t.element_size() for t in (w.kv, w.q_g, w.q_l, w.z_off))
+    need_flush = in_bytes < 4 * L2_BYTES
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if need_flush else None
+    stream = torch.cuda.current_stream()
+
+    def step(ev=None):
+        if ev: ev[0].record(stream)
+        ctx.rk_mla_online_attn(req, w.kv, w.q_g, None, bufs["O_g"], bufs["lse_g"], None, None)
+        if ev: ev[1].record(stream)
+        ctx.rk_mla_online_attn(req, w.kv, None, w.q_l, None, None, bufs["O_l"], bufs["lse_l"])
+        if ev: ev[2].record(stream)
+        ctx.rk_group_sliced_proj(req, bufs["O_g"], bufs["O_l"], w.w_uv, w.w_a, bufs["z_on_g"], bufs["z_on_l"],
+                                 bufs["workspace"])
+        ctx.rk_combine_offline(req, bufs["z_on_g"], bufs["z_on_l"], w.z_off, w.w_b, bufs["z"], bufs["y"])
+        if ev: ev[3].record(stream)
+
+    launches_per_step = 2 + 4 + 1 + 1   # attention x2, projection GEMMs x4, combine, W_b GEMM
+
+    for _ in range(args.warmup):
+        step()
+        if need_flush: flush_buf.fill_(1)
+    torch.cuda.synchronize()
+    ctx.rk_poll_status()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    if world > 1: dist.barrier()
+    torch.cuda.synchronize()
+    for i in range(args.steps):
+        step(evs[i])
+        if need_flush: flush_buf.fill_(1)
+    torch.cuda.synchronize()
+    if world > 1: dist.barrier()
+    sampler.stop_flag = True
+    ctx.rk_poll_status()
+    step_ms = [evs[i][0].elapsed_time(evs[i][3]) for i in range(args.steps)]
+    attn_ms = [evs[i][0].elapsed_time(evs[i][2]) for i in range(args.steps)]
+    attn_g_ms = [evs[i][0].elapsed_time(evs[i][1]) for i in range(args.steps)]
+    rest_ms = [evs[i][2].elapsed_time(evs[i][3]) for i in range(args.steps)]
+    total_ms = float(sum(step_ms))
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1: dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max = float(t.item())
+    sampler.join(timeout=2)
+    clocks = sampler.summary()
+
+    # end to end through the host-buffer entry point (H2D of the request inputs + D2H of y per step)
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda x: x.to("cpu").pin_memory()
+        hk, hqg, hql, hzo = pin(w.kv), pin(w.q_g), pin(w.q_l), pin(w.z_off)
+        y_h = torch.empty((req.T, prof.d_model), dtype=torch.bfloat16).pin_memory()
+        ctx.rk_layer_host(req, hk, hqg, hql, hzo, w.w_uv, w.w_a, w.w_b, bufs, y_h)   # warm-up
+        if world > 1: dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            ctx.rk_layer_host(req, hk, hqg, hql, hzo, w.w_uv, w.w_a, w.w_b, bufs, y_h)
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0)
+        te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        if world > 1: dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        ctx.rk_poll_status()
+        e2e = dict(value=world * req.T * args.e2e_steps / float(te.item()), unit="tokens/s",
+                   h2d_bytes_per_step=int(in_bytes), d2h_bytes_per_step=int(y_h.numel() * 2),
+                   ms_per_step=float(te.item()) * 1e3 / args.e2e_steps)
+        del hk, hqg, hql, hzo
+
+    if rank != 0:
+        if world > 1: dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    attn_tflops = fl_attn / (np.mean(attn_ms) * 1e-3) / 1e12
+    roofline = dict(bound="tensor", kernel="rk_mla_attn_kernel (Global + Local launches)",
+                    achieved=attn_tflops, peak=peaks["bf16_sustained"], unit="TFLOP/s",
+                    frac=attn_tflops / peaks["bf16_sustained"], peak_source=peaks["source"] + " sustained bf16",
+                    frac_of_burst=attn_tflops / peaks["bf16_burst"], frac_of_nominal=attn_tflops / 2250.0,
+                    launches_per_step=2, ms_per_step=float(np.mean(attn_ms)),
+                    ms_global_pass=float(np.mean(attn_g_ms)), traffic=None)
+    rest_tflops = (fl_proj + fl_wb) / (np.mean(rest_ms) * 1e-3) / 1e12
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        rows = pick_oracle_rows(w, args.oracle_pairs)
+        dt, pairs, out = oracle_sample_run(w, rows)
+        allp = total_pairs(prof, req)
+        # while the sample is at hand: parity of this very run against the checker
+        from tests.helpers import rel_l2
+        y_gpu = bufs["y"][torch.as_tensor(rows, device=dev)].float().cpu().numpy().astype(np.float64)
+        cpu_baseline = dict(value=req.T / (dt * allp / pairs), unit="tokens/s", cores=os.cpu_count(), kind="oracle",
+                            threads=torch.get_num_threads(),
+                            sample=f"{len(rows)} seeded rows, {pairs} of {allp} visible (row,key,head) pairs in "
+                                   f"{dt:.1f} s, extrapolated by pair count",
+                            pairs_per_s=pairs / dt, parity_rel_l2_y=rel_l2(y_gpu, out["y"]))
+
+    line = dict(metric="mla_online_prefill_tokens_per_s_per_layer", value=world * req.T * args.steps / (total_ms_max * 1e-3),
+                unit="tokens/s", n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=total_ms_max / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="bf16", data="synthetic",
+                config=dict(workload=name, regime=args.regime, T=req.T, n_prot=req.A, n_segs=lay.n_segs,
+                            heads=prof.n_heads, groups=prof.n_groups, o_rank=prof.o_rank, d_model=prof.d_model,
+                            l2="inputs larger than L2" if not need_flush else "L2 flushed between iterations",
+                            flops_attn=fl_attn, flops_proj=fl_proj + fl_wb),
+                clocks=clocks, e2e=e2e, gpu_launches=launches_per_step * args.steps, roofline=roofline,
+                proj_tflops=rest_tflops, proj_ms_per_step=float(np.mean(rest_ms)), cpu_baseline=cpu_baseline)
+    print(json.dumps(line))
+    if world > 1: dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

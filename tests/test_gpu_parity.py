@@ -81,7 +81,13 @@ def test_segmented_merge(rk, dtype, P):
 
 # -- (2) attention -----------------------------------------------------------------------------------
 
-def check_attention(rk, w, rows=None):
+# lse tolerance: the rotated rope sub-vector is rounded to bf16 once more before QK^T, which moves a
+# logit by about |q_rope| |k_rope| sm_scale 2^-9 ~ 1e-3 when q, k are O(1) ("sharp" values) and by
+# far less for the benchmark's N(0, 0.02) latents; lse is a convex combination of logits.
+LSE_TOL = {"mandated": 1e-3, "sharp": 5e-3}
+
+
+def check_attention(rk, w, rows=None, lse_tol=LSE_TOL["sharp"]):
     ctx, req = make(rk, w)
     T = w.layout.n_rows
     rows = np.arange(T) if rows is None else rows
@@ -90,17 +96,17 @@ def check_attention(rk, w, rows=None):
     O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
     ctx.rk_poll_status()
     r1 = assert_close(f64(O_g)[rows], exp["O_g"], "O_g")
-    assert max_abs(f64(lse_g)[rows], exp["lse_g"]) <= 1e-3
+    assert max_abs(f64(lse_g)[rows], exp["lse_g"]) <= lse_tol
     inv = oracle.inverse_row_map(w.prot_rows, T)
     slots = inv[rows][inv[rows] >= 0]
     r2 = assert_close(f64(O_l)[slots], exp["O_l"], "O_l")
-    assert max_abs(f64(lse_l)[slots], exp["lse_l"]) <= 1e-3
+    assert max_abs(f64(lse_l)[slots], exp["lse_l"]) <= lse_tol
     return r1, r2
 
 
 @pytest.mark.parametrize("regime", ["mandated", "sharp"])
 def test_attention_tiny(rk, regime):
-    check_attention(rk, synth.make_workload("tiny", regime=regime))
+    check_attention(rk, synth.make_workload("tiny", regime=regime), lse_tol=LSE_TOL[regime])
 
 
 @pytest.mark.parametrize("seed", [5, 6])
