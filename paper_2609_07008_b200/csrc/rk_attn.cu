@@ -14,8 +14,9 @@
 // each CTA streams its 128 keys of the tile, for PV its 128 of each 256 output dims.  The same
 // [128 keys x 64 dims] 128B-swizzled TMA box serves as K-major B (QK^T) and MN-major B (PV).
 //
-// Warp roles per CTA (256 threads): warp 0 TMA producer, warp 1 UMMA issuer (leader CTA only),
-// warp 2 query relocation, warps 4-7 softmax / correction / epilogue (thread <-> TMEM lane).
+// Warp roles per CTA (384 threads): warp 0 TMA producer, warp 1 UMMA issuer (leader CTA only),
+// warp 2 query relocation, warps 4-11 softmax / correction / epilogue (two warps per TMEM lane
+// quarter, each owning half of the columns).
 #include <cuda_bf16.h>
 
 #include "rk_internal.h"
@@ -23,8 +24,10 @@
 namespace rk {
 namespace {
 
-constexpr int kRing = 6;
+constexpr int kAttnThreads = 384;       // 4 role warps + 8 softmax warps
+constexpr int kStages = 3;                // ring of 32 KB stages (two 16 KB TMA boxes each)
 constexpr uint32_t kChunkBytes = 16384;  // 128 keys x 64 dims bf16
+constexpr uint32_t kStageBytes = 2 * kChunkBytes;
 constexpr uint32_t kQChunkBytes = 8192;  // 64 rows x 64 dims bf16
 
 // shared memory map (offsets from a 1024-byte aligned base)
@@ -33,15 +36,15 @@ constexpr uint32_t kOffQPristine = kOffQLat + 8 * kQChunkBytes;  // rope chunk a
 constexpr uint32_t kOffQRot = kOffQPristine + kQChunkBytes;      // 2 rotated rope chunks
 constexpr uint32_t kOffP = kOffQRot + 2 * kQChunkBytes;          // 4 sub-chunks [64 x 64 keys]
 constexpr uint32_t kOffRing = kOffP + 4 * kQChunkBytes;
-constexpr uint32_t kOffBars = kOffRing + kRing * kChunkBytes;
+constexpr uint32_t kOffBars = kOffRing + kStages * kStageBytes;
 // barrier indices (8 bytes each)
 constexpr int kBarQFull = 0, kBarQFree = 1, kBarQrReady = 2 /*2*/, kBarQrFree = 4 /*2*/, kBarRingFull = 6,
-              kBarRingEmpty = kBarRingFull + kRing, kBarSFull = kBarRingEmpty + kRing /*2*/,
+              kBarRingEmpty = kBarRingFull + kStages, kBarSFull = kBarRingEmpty + kStages /*2*/,
               kBarPReady = kBarSFull + 2, kBarPvDone = kBarPReady + 1, kNumBars = kBarPvDone + 1;
 constexpr uint32_t kOffTmemPtr = kOffBars + kNumBars * 8;
 constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
-constexpr uint32_t kOffXchg = kOffAbort + 8;                 // u64 [2 parity][2 halves][64]: (seq << 32) | value
-constexpr uint32_t kSmemUsed = kOffXchg + 2 * 2 * 64 * 8;
+constexpr uint32_t kOffXchg = kOffAbort + 8;                 // u64 [2 parity][4 parts][64]: (seq << 32) | value
+constexpr uint32_t kSmemUsed = kOffXchg + 2 * 4 * 64 * 8;
 constexpr uint32_t kSmemBytes = kSmemUsed + 1024;            // + alignment slack
 
 // TMEM columns
@@ -72,49 +75,73 @@ struct SegIter {
   }
 };
 
-// Ring bookkeeping shared by the producer and the UMMA issuer: both walk the same slot
-// sequence.  A V stage needs two consecutive slots (fixed 16 KB apart for the descriptor's
-// leading byte offset), so a pair never starts on the last slot: that slot is skipped.
+// Ring bookkeeping shared by the producer and the UMMA issuer: both walk the same stage
+// sequence.  A stage holds two 16 KB boxes: two 64-dim K chunks (QK^T), the single rope chunk,
+// or the two 64-dim halves of this CTA's 128 output dims (PV; 16 KB apart = the descriptor's
+// leading byte offset).
 struct RingPos {
-  uint32_t slot = 0;
-  uint32_t phases = 0;  // bit s = parity to wait for on slot s
-  __device__ void advance() { phases ^= (1u << slot); slot = (slot + 1 == kRing) ? 0 : slot + 1; }
-  __device__ void skip() { slot = (slot + 1 == kRing) ? 0 : slot + 1; }
-  __device__ uint32_t parity() const { return (phases >> slot) & 1u; }
+  uint32_t it = 0;  // stages used so far
+  __device__ uint32_t stage() const { return it % kStages; }
+  __device__ uint32_t parity() const { return (it / kStages) & 1u; }
+  __device__ void advance() { ++it; }
 };
 
-// The two threads that hold the two halves of one query row (lanes m and m + 64 of TMEM, in
-// different warps) swap one float through shared memory.  Sequence-tagged and double-buffered
-// by sequence parity; the poll is bounded like every other wait in this kernel.
-__device__ __forceinline__ bool pair_exchange(volatile unsigned long long* xbuf, int kh, int m, uint32_t seq,
-                                              float mine, float& other, uint64_t limit_ns,
+// number of key tiles a row tile walks through (all visible segments)
+__device__ __forceinline__ int count_key_tiles(const AttnParams& p, int maxpos) {
+  SegIter it(p, maxpos);
+  int n = 0;
+  while (it.next()) n += (it.kmax + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
+  return n;
+}
+
+// The four threads that share one query row (TMEM lanes m and m + 64, two column halves each,
+// all in different warps) combine one float through shared memory.  Sequence-tagged and
+// double-buffered by sequence parity; the poll is bounded like every other wait here.
+template <bool kMax>
+__device__ __forceinline__ bool quad_exchange(volatile unsigned long long* xbuf, int part, int m, uint32_t seq,
+                                              float mine, float& combined, uint64_t limit_ns,
                                               volatile int* abort_flag, DeviceStatus* st, int aux) {
-  volatile unsigned long long* base = xbuf + (seq & 1u) * 128;
-  base[kh * 64 + m] = ((unsigned long long)seq << 32) | (unsigned long long)__float_as_uint(mine);
-  volatile unsigned long long* theirs = base + (kh ^ 1) * 64 + m;
-  uint64_t t0 = 0;
-  uint32_t spins = 0;
-  while (true) {
-    const unsigned long long v = *theirs;
-    if ((uint32_t)(v >> 32) == seq) {
-      other = __uint_as_float((uint32_t)v);
-      return true;
-    }
-    if ((++spins & 0xff) == 0) {
-      if (*abort_flag != 0) return false;
-      if (t0 == 0) t0 = globaltimer_ns();
-      if (globaltimer_ns() - t0 > limit_ns) {
-        *abort_flag = 1;
-        report_timeout(st, 20, aux);
-        return false;
+  volatile unsigned long long* base = xbuf + (seq & 1u) * 256;
+  base[part * 64 + m] = ((unsigned long long)seq << 32) | (unsigned long long)__float_as_uint(mine);
+  float acc = mine;
+#pragma unroll
+  for (int o = 1; o < 4; ++o) {
+    volatile unsigned long long* theirs = base + ((part + o) & 3) * 64 + m;
+    uint64_t t0 = 0;
+    uint32_t spins = 0;
+    while (true) {
+      const unsigned long long v = *theirs;
+      if ((uint32_t)(v >> 32) == seq) {
+        const float x = __uint_as_float((uint32_t)v);
+        acc = kMax ? fmaxf(acc, x) : acc + x;
+        break;
+      }
+      if ((++spins & 0xff) == 0) {
+        if (*abort_flag != 0) return false;
+        if (t0 == 0) t0 = globaltimer_ns();
+        if (globaltimer_ns() - t0 > limit_ns) {
+          *abort_flag = 1;
+          report_timeout(st, 20, aux);
+          return false;
+        }
       }
     }
   }
+  combined = acc;
+  return true;
+}
+#define quad_exchange_max quad_exchange<true>
+#define quad_exchange_sum quad_exchange<false>
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
 }  // namespace
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     rk_mla_attn_kernel(const __grid_constant__ AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -130,7 +157,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + kOffTmemPtr);
   const uint64_t limit = p.wait_ns;
 
-  if (threadIdx.x < 256) reinterpret_cast<volatile unsigned long long*>(smem + kOffXchg)[threadIdx.x] = 0ull;
+  for (int i = threadIdx.x; i < 512; i += kAttnThreads) reinterpret_cast<volatile unsigned long long*>(smem + kOffXchg)[i] = 0ull;
   if (threadIdx.x == 0) {
     *abort_flag = 0;
     mbar_init(bar(kBarQFull), 1);
@@ -140,11 +167,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
       mbar_init(bar(kBarQrFree + b), 1);
       mbar_init(bar(kBarSFull + b), 1);
     }
-    for (int s = 0; s < kRing; ++s) {
+    for (int s = 0; s < kStages; ++s) {
       mbar_init(bar(kBarRingFull + s), 1);
       mbar_init(bar(kBarRingEmpty + s), 1);
     }
-    mbar_init(bar(kBarPReady), 8);
+    mbar_init(bar(kBarPReady), 16);
     mbar_init(bar(kBarPvDone), 1);
     fence_mbar_init_cluster();
   }
@@ -162,87 +189,97 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
 
   // =====================================================================================
   if (warp == 0) {
-    // ------------------------------ TMA producer -----------------------------------------
+    // ------------------------------ TMA producer (whole warp loops; one elected lane issues) ------
     if (lane == 0) {
       tma_prefetch_desc(&p.tm_q);
       tma_prefetch_desc(&p.tm_kv);
-      RingPos rp;
-      uint32_t qfree_phase = 0;
-      uint32_t used_slots = 0;  // bit s set once slot s has been filled at least once
-      bool ok = true;
-      int n_done = 0;
-      for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs, ++n_done) {
-        const AttnWorkItem item = p.work[w];
-        // Q tile: wait until the previous tile's QK^T MMAs have finished reading it
-        if (n_done > 0) {
-          ok = mbar_wait_bounded<true>(bar(kBarQFree), qfree_phase, limit, abort_flag, p.status, W_QFREE, w);
-          qfree_phase ^= 1;
-          if (!ok) break;
+    }
+    RingPos rp;
+    uint32_t qfree_phase = 0;
+    bool ok = true;
+    int n_done = 0;
+    // fills one stage with one or two boxes; every lane waits, one lane issues
+    auto fill = [&](int col0, int col1, int row, int w) -> bool {
+      const uint32_t s = rp.stage();
+      if (rp.it >= (uint32_t)kStages) {
+        if (!mbar_wait_bounded<false>(bar(kBarRingEmpty + s), rp.parity() ^ 1u, limit, abort_flag, p.status,
+                                      W_RINGEMPTY, w))
+          return false;
+      }
+      if (elect_one()) {
+        const uint32_t full_local = bar(kBarRingFull + s);
+        const uint32_t nbox = (col1 >= 0) ? 2u : 1u;
+        if (p.debug & 2) {
+          if (leader) mbar_arrive(full_local);
+        } else {
+          if (leader) mbar_arrive_expect_tx(full_local, 2 * nbox * kChunkBytes);
+          const uint32_t full_remote = mapa_shared(full_local, 0);
+          const uint32_t dst = smem_base + kOffRing + s * kStageBytes;
+          tma_load_2d_pair(dst, &p.tm_kv, full_remote, col0, row);
+          if (col1 >= 0) tma_load_2d_pair(dst + kChunkBytes, &p.tm_kv, full_remote, col1, row);
         }
+      }
+      __syncwarp();
+      rp.advance();
+      return true;
+    };
+    auto load_k = [&](int seg_row0, int kb, int w) -> bool {  // this CTA's 128 keys: 4 dim pairs + rope
+      const int row = seg_row0 + kb + (int)crank * 128;
+      for (int d = 0; d < 4; ++d)
+        if (!fill(128 * d, 128 * d + 64, row, w)) return false;
+      return fill(kDLatent, -1, row, w);
+    };
+    auto load_v = [&](int seg_row0, int kb, int w) -> bool {  // (key half, output half): this CTA's 128 dims
+      for (int kh = 0; kh < 2; ++kh)
+        for (int h = 0; h < 2; ++h) {
+          const int col = 256 * h + 128 * (int)crank;
+          if (!fill(col, col + 64, seg_row0 + kb + kh * 128, w)) return false;
+        }
+      return true;
+    };
+    for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs, ++n_done) {
+      const AttnWorkItem item = p.work[w];
+      // Q tile: wait until the previous tile's QK^T MMAs have finished reading it
+      if (n_done > 0) {
+        ok = mbar_wait_bounded<false>(bar(kBarQFree), qfree_phase, limit, abort_flag, p.status, W_QFREE, w);
+        qfree_phase ^= 1;
+        if (!ok) break;
+      }
+      if (elect_one()) {
         mbar_arrive_expect_tx(bar(kBarQFull), 9 * kQChunkBytes);
         const int qrow = item.tile * kAttnRowsPerPair + (int)crank * kAttnRowsPerCta;
         for (int d = 0; d < 9; ++d)
           tma_load_2d(smem_base + kOffQLat + d * kQChunkBytes, &p.tm_q, bar(kBarQFull), d * 64, qrow);
-
-        auto load_slot = [&](int col, int row) -> bool {
-          if (used_slots & (1u << rp.slot)) {
-            if (!mbar_wait_bounded<true>(bar(kBarRingEmpty + rp.slot), rp.parity() ^ 1u, limit, abort_flag,
-                                         p.status, W_RINGEMPTY, w))
-              return false;
-          }
-          used_slots |= (1u << rp.slot);
-          const uint32_t full_local = bar(kBarRingFull + rp.slot);
-          if (leader) mbar_arrive_expect_tx(full_local, 2 * kChunkBytes);
-          tma_load_2d_pair(smem_base + kOffRing + rp.slot * kChunkBytes, &p.tm_kv, mapa_shared(full_local, 0), col,
-                           row);
-          rp.advance();
-          return true;
-        };
-        auto load_k = [&](int seg_row0, int kb) -> bool {  // 9 single slots: this CTA's 128 keys
-          const int row = seg_row0 + kb + (int)crank * 128;
-          for (int d = 0; d < 9; ++d)
-            if (!load_slot(d * 64, row)) return false;
-          return true;
-        };
-        auto load_v = [&](int seg_row0, int kb) -> bool {  // 4 pairs: (key half, output half)
-          for (int kh = 0; kh < 2; ++kh)
-            for (int h = 0; h < 2; ++h) {
-              if (rp.slot == kRing - 1) rp.skip();
-              const int row = seg_row0 + kb + kh * 128;
-              const int col = 256 * h + 128 * (int)crank;
-              if (!load_slot(col, row)) return false;
-              if (!load_slot(col + 64, row)) return false;
-            }
-          return true;
-        };
-
-        // order of consumption: K(0), K(1), V(0), K(2), V(1), ..., V(last)
-        SegIter it(p, item.maxpos);
-        int prev_row0 = -1, prev_kb = 0;
-        while (ok && it.next()) {
-          const int row0 = p.seg_off[it.seg];
-          for (int kb = 0; kb < it.kmax && ok; kb += kAttnKeysPerTile) {
-            ok = load_k(row0, kb);
-            if (ok && prev_row0 >= 0) ok = load_v(prev_row0, prev_kb);
-            prev_row0 = row0;
-            prev_kb = kb;
-          }
-        }
-        if (ok && prev_row0 >= 0) ok = load_v(prev_row0, prev_kb);
       }
-      // drain: every slot this CTA filled must have been released by the tensor core, and the
-      // last Q tile must be free, before the CTA may exit
-      if (ok && n_done > 0)
-        ok = mbar_wait_bounded<true>(bar(kBarQFree), qfree_phase, limit, abort_flag, p.status, W_DRAIN, -1);
-      for (int s = 0; s < kRing && ok; ++s) {
-        if (used_slots & (1u << s))
-          ok = mbar_wait_bounded<true>(bar(kBarRingEmpty + s), ((rp.phases >> s) & 1u) ^ 1u, limit, abort_flag,
-                                       p.status, W_DRAIN, s);
+      __syncwarp();
+      // order of consumption: K(0), K(1), V(0), K(2), V(1), ..., V(last)
+      SegIter it(p, item.maxpos);
+      int prev_row0 = -1, prev_kb = 0;
+      while (ok && it.next()) {
+        const int row0 = p.seg_off[it.seg];
+        for (int kb = 0; kb < it.kmax && ok; kb += kAttnKeysPerTile) {
+          ok = load_k(row0, kb, w);
+          if (ok && prev_row0 >= 0) ok = load_v(prev_row0, prev_kb, w);
+          prev_row0 = row0;
+          prev_kb = kb;
+        }
+      }
+      if (ok && prev_row0 >= 0) ok = load_v(prev_row0, prev_kb, w);
+    }
+    // drain: every stage this CTA filled must have been released by the tensor core, and the
+    // last Q tile must be free, before the CTA may exit
+    if (ok && n_done > 0)
+      ok = mbar_wait_bounded<false>(bar(kBarQFree), qfree_phase, limit, abort_flag, p.status, W_DRAIN, -1);
+    for (uint32_t back = 1; back <= (uint32_t)kStages && ok; ++back) {
+      if (rp.it >= back) {
+        const uint32_t u = rp.it - back;  // a fill that has not been waited for yet
+        ok = mbar_wait_bounded<false>(bar(kBarRingEmpty + u % kStages), (u / kStages) & 1u, limit, abort_flag,
+                                      p.status, W_DRAIN, (int)u);
       }
     }
   } else if (warp == 1) {
-    // ------------------------------ UMMA issuer (leader CTA) --------------------------------
-    if (leader && lane == 0) {
+    // ------------------------------ UMMA issuer (leader CTA; whole warp loops, elected lane issues) --
+    if (leader) {
       RingPos rp;
       uint32_t qr_ready_phase[2] = {0, 0};
       uint32_t p_ready_phase = 0;
@@ -253,8 +290,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
 
       for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
         const AttnWorkItem item = p.work[w];
-        int kt_issued = 0;   // key tiles whose QK^T has been issued
-        int kt_pv = 0;       // key tiles whose PV has been issued
+        const int n_kt = count_key_tiles(p, item.maxpos);
+        int kt_issued = 0;  // key tiles whose QK^T has been issued
+        int kt_pv = 0;      // key tiles whose PV has been issued
 
         auto issue_qk = [&](bool first_of_seg, bool last_of_seg, uint32_t rb) -> bool {
           if (first_of_seg) {
@@ -264,23 +302,39 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
             qr_ready_phase[rb] ^= 1;
           }
           const uint32_t tmem_s = tmem_base + kColS + (uint32_t)(kt_issued & 1) * 128u;
-          for (int d = 0; d < 9; ++d) {
-            if (!mbar_wait_bounded<true>(bar(kBarRingFull + rp.slot), rp.parity(), limit, abort_flag, p.status,
-                                         W_RINGFULL, w))
+#pragma unroll 1
+          for (int st = 0; st < 5; ++st) {
+            const uint32_t s = rp.stage();
+            if (!mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
               return false;
-            tc_fence_after_sync();
-            const uint32_t a_addr = (d < 8) ? (q_base + d * kQChunkBytes) : (smem_base + kOffQRot + rb * kQChunkBytes);
-            const uint32_t b_addr = smem_base + kOffRing + rp.slot * kChunkBytes;
+            const uint32_t b_addr = smem_base + kOffRing + s * kStageBytes;
+            if (elect_one()) {
+              if (st < 4) {
+                const uint32_t a_addr = q_base + 2 * st * kQChunkBytes;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              umma_f16<2>(tmem_s, umma_desc_sw128(a_addr + k * 32, 16, 1024), umma_desc_sw128(b_addr + k * 32, 16, 1024),
-                          kIdescQK, (d > 0 || k > 0) ? 1u : 0u);
+                for (int k = 0; k < 8; ++k) {
+                  umma_f16<2>(tmem_s, umma_desc_sw128(a_addr + (k >> 2) * kQChunkBytes + (k & 3) * 32, 16, 1024),
+                              umma_desc_sw128(b_addr + (k >> 2) * kChunkBytes + (k & 3) * 32, 16, 1024), kIdescQK,
+                              (st > 0 || k > 0) ? 1u : 0u);
+                }
+                umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
+              } else {
+                const uint32_t a_addr = smem_base + kOffQRot + rb * kQChunkBytes;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  umma_f16<2>(tmem_s, umma_desc_sw128(a_addr + k * 32, 16, 1024),
+                              umma_desc_sw128(b_addr + k * 32, 16, 1024), kIdescQK, 1u);
+                }
+                umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
+                umma_commit_2_mc(bar(kBarSFull + (kt_issued & 1)), 3);
+                if (last_of_seg) umma_commit_2_mc(bar(kBarQrFree + rb), 3);
+                // all QK^T of this row tile issued: the Q tile is free once they complete
+                if (kt_issued + 1 == n_kt) umma_commit_2_mc(bar(kBarQFree), 3);
+              }
             }
-            umma_commit_2_mc(bar(kBarRingEmpty + rp.slot), 3);
+            __syncwarp();
             rp.advance();
           }
-          umma_commit_2_mc(bar(kBarSFull + (kt_issued & 1)), 3);
-          if (last_of_seg) umma_commit_2_mc(bar(kBarQrFree + rb), 3);
           ++kt_issued;
           return true;
         };
@@ -289,21 +343,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
             return false;
           p_ready_phase ^= 1;
           tc_fence_after_sync();
-          for (int kh = 0; kh < 2; ++kh)
-            for (int h = 0; h < 2; ++h) {
-              if (rp.slot == kRing - 1) rp.skip();
-              const uint32_t s0 = rp.slot;
-              if (!mbar_wait_bounded<true>(bar(kBarRingFull + s0), rp.parity(), limit, abort_flag, p.status,
-                                           W_RINGFULL, w))
-                return false;
-              rp.advance();
-              if (!mbar_wait_bounded<true>(bar(kBarRingFull + s0 + 1), rp.parity(), limit, abort_flag, p.status,
-                                           W_RINGFULL, w))
-                return false;
-              rp.advance();
-              tc_fence_after_sync();
-              const uint32_t b_addr = smem_base + kOffRing + s0 * kChunkBytes;
-              const uint32_t tmem_o = tmem_base + kColO + (uint32_t)h * 128u;
+#pragma unroll 1
+          for (int q = 0; q < 4; ++q) {
+            const int kh = q >> 1, h = q & 1;
+            const uint32_t s = rp.stage();
+            if (!mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
+              return false;
+            const uint32_t b_addr = smem_base + kOffRing + s * kStageBytes;
+            const uint32_t tmem_o = tmem_base + kColO + (uint32_t)h * 128u;
+            if (elect_one()) {
 #pragma unroll
               for (int k = 0; k < 8; ++k) {
                 const uint32_t a_addr = p_base + (2 * kh + (k >> 2)) * kQChunkBytes + (k & 3) * 32;
@@ -311,10 +359,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
                             umma_desc_sw128(b_addr + k * 2048, kChunkBytes, 1024), kIdescPV,
                             (kt_pv > 0 || kh > 0 || k > 0) ? 1u : 0u);
               }
-              umma_commit_2_mc(bar(kBarRingEmpty + s0), 3);
-              umma_commit_2_mc(bar(kBarRingEmpty + s0 + 1), 3);
+              umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
+              if (q == 3) umma_commit_2_mc(bar(kBarPvDone), 3);
             }
-          umma_commit_2_mc(bar(kBarPvDone), 3);
+            __syncwarp();
+            rp.advance();
+          }
           ++kt_pv;
           return true;
         };
@@ -330,8 +380,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
             if (ok && kt_issued >= 2) ok = issue_pv();
           }
         }
-        // all QK^T of this row tile issued: the Q tile is free once they complete
-        if (ok) umma_commit_2_mc(bar(kBarQFree), 3);
         while (ok && kt_pv < kt_issued) ok = issue_pv();
       }
     }
@@ -392,12 +440,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
     }
   } else if (warp >= 4) {
     // ------------------------------ softmax / correction / epilogue ----------------------------
-    const int L = threadIdx.x - 128;  // TMEM lane
-    const int m = L & 63;             // row within this CTA
-    const int kh = L >> 6;            // which 128-key half of the tile (and which dims half of O)
-    const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
+    // 8 warps.  Warp sw = warp - 4 reads TMEM lanes [32 (sw % 4), +32) and the column half
+    // ch = sw / 4 of every 128-column buffer, so one query row (TMEM lanes m and m + 64) is
+    // shared by four threads: (kh, ch) = (key half of the tile, 64-key quarter within it).
+    const int sw = warp - 4;
+    const int ch = sw >> 2;
+    const int L = (sw & 3) * 32 + lane;  // TMEM lane
+    const int m = L & 63;                // row within this CTA
+    const int kh = L >> 6;               // which 128-key half of the tile (and which dims half of O)
+    const int part = kh * 2 + ch;        // which 64-key quarter of the tile
+    const uint32_t lane_base = ((uint32_t)((sw & 3) * 32)) << 16;
     volatile unsigned long long* xbuf = reinterpret_cast<volatile unsigned long long*>(smem + kOffXchg);
-    uint32_t xseq = 0;  // exchange sequence number (warps {4,6} and {5,7} hold the halves of the same rows)
+    uint32_t xseq = 0;  // exchange sequence number
     uint32_t s_full_phase[2] = {0, 0};
     uint32_t pv_done_phase = 0;
     bool ok = true;
@@ -420,78 +474,102 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
       SegIter it(p, item.maxpos);
       while (ok && it.next()) {
         const int n_seg = p.seg_off[it.seg + 1] - p.seg_off[it.seg];
-        int lim = pos - p.seg_delta[it.seg];           // last visible canonical index
+        int lim = pos - p.seg_delta[it.seg];  // last visible canonical index
         if (lim > n_seg - 1) lim = n_seg - 1;
         if (pos < 0) lim = -1;
         for (int kb = 0; kb < it.kmax && ok; kb += kAttnKeysPerTile, ++kt) {
-          int nv = lim - (kb + kh * 128) + 1;
-          nv = nv < 0 ? 0 : (nv > 128 ? 128 : nv);
+          int nv = lim - (kb + part * 64) + 1;
+          nv = nv < 0 ? 0 : (nv > 64 ? 64 : nv);
           const int b = kt & 1;
-          ok = mbar_wait_bounded<true>(bar(kBarSFull + b), s_full_phase[b], limit, abort_flag, p.status, W_SFULL, w);
+          ok = mbar_wait_bounded<false>(bar(kBarSFull + b), s_full_phase[b], limit, abort_flag, p.status, W_SFULL, w);
           s_full_phase[b] ^= 1;
           if (!ok) break;
           tc_fence_after_sync();
-          uint32_t s[128];
-          const uint32_t taddr = tmem_base + lane_base + kColS + (uint32_t)b * 128u;
+          if (p.debug & 1) {
+            if (kt > 0) {
+              ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
+              pv_done_phase ^= 1;
+              if (!ok) break;
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(p_ready_remote);
+            continue;
+          }
+          uint32_t s[64];
+          const uint32_t taddr = tmem_base + lane_base + kColS + (uint32_t)b * 128u + (uint32_t)ch * 64u;
           tmem_ld_x32(taddr + 0, s + 0);
           tmem_ld_x32(taddr + 32, s + 32);
-          tmem_ld_x32(taddr + 64, s + 64);
-          tmem_ld_x32(taddr + 96, s + 96);
           tmem_wait_ld();
-          float mx = -INFINITY;
+          const bool full = __all_sync(0xffffffffu, nv == 64);  // no masking needed anywhere in this warp
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          if (full) {
 #pragma unroll
-          for (int c = 0; c < 128; ++c) {
-            const float v = (c < nv) ? __uint_as_float(s[c]) : -INFINITY;
-            mx = fmaxf(mx, v);
+            for (int c = 0; c < 64; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(s[c]));
+          } else {
+#pragma unroll
+            for (int c = 0; c < 64; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], (c < nv) ? __uint_as_float(s[c]) : -INFINITY);
           }
-          float mx_other;
-          ok = pair_exchange(xbuf, kh, m, ++xseq, mx, mx_other, limit, abort_flag, p.status, w);
+          const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+          float mxo = mx;
+          if (!(p.debug & 4)) ok = quad_exchange_max(xbuf, part, m, ++xseq, mx, mxo, limit, abort_flag, p.status, w);
           if (!ok) break;
-          const float mt = fmaxf(mx, mx_other) * scale;
+          const float mt = mxo * scale;
           // lazy rescale: only when the running maximum grows by more than 2^8
           float alpha = 1.f;
           bool need = false;
           if (mt > m_run + 8.f) {  // also true for the first finite maximum (m_run = -inf)
-            alpha = (m_run == -INFINITY) ? 0.f : exp2f(m_run - mt);
+            alpha = (m_run == -INFINITY) ? 0.f : fast_exp2(m_run - mt);
             need = (m_run != -INFINITY);
             m_run = mt;
             l_run *= alpha;
           }
           const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-          uint32_t pk[64];
-          float lsum = 0.f;
+          uint32_t pk[32];
+          float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+          if (full) {
 #pragma unroll
-          for (int c = 0; c < 128; c += 2) {
-            float p0 = (c < nv) ? exp2f(fmaf(__uint_as_float(s[c]), scale, -m_use)) : 0.f;
-            float p1 = (c + 1 < nv) ? exp2f(fmaf(__uint_as_float(s[c + 1]), scale, -m_use)) : 0.f;
-            lsum += p0 + p1;
-            pk[c >> 1] = pack_bf16(p0, p1);
+            for (int c = 0; c < 64; c += 2) {
+              const float p0 = fast_exp2(fmaf(__uint_as_float(s[c]), scale, -m_use));
+              const float p1 = fast_exp2(fmaf(__uint_as_float(s[c + 1]), scale, -m_use));
+              ls4[(c >> 1) & 3] += p0 + p1;
+              pk[c >> 1] = pack_bf16(p0, p1);
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 64; c += 2) {
+              const float p0 = (c < nv) ? fast_exp2(fmaf(__uint_as_float(s[c]), scale, -m_use)) : 0.f;
+              const float p1 = (c + 1 < nv) ? fast_exp2(fmaf(__uint_as_float(s[c + 1]), scale, -m_use)) : 0.f;
+              ls4[(c >> 1) & 3] += p0 + p1;
+              pk[c >> 1] = pack_bf16(p0, p1);
+            }
           }
-          l_run += lsum;
+          l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
           // P buffer and O are free once the previous PV has completed
           if (kt > 0) {
-            ok = mbar_wait_bounded<true>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
+            ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
             pv_done_phase ^= 1;
             if (!ok) break;
             tc_fence_after_sync();
             if (__any_sync(0xffffffffu, need)) {
 #pragma unroll 1
-              for (int cc = 0; cc < 256; cc += 32) {
+              for (int cc = 0; cc < 128; cc += 32) {  // this thread's 2 x 64 columns of O
                 uint32_t o[32];
-                tmem_ld_x32(tmem_base + lane_base + kColO + cc, o);
+                const uint32_t oaddr = tmem_base + lane_base + kColO + (uint32_t)((cc >> 6) * 128 + ch * 64 + (cc & 63));
+                tmem_ld_x32(oaddr, o);
                 tmem_wait_ld();
 #pragma unroll
                 for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                tmem_st_x32(tmem_base + lane_base + kColO + cc, o);
+                tmem_st_x32(oaddr, o);
               }
               tmem_wait_st();
             }
           }
-          // write P (bf16, K-major 128B swizzle): row m, sub-chunks 2kh and 2kh+1
-          uint8_t* pbase = smem + kOffP + (2 * kh) * kQChunkBytes;
+          // write P (bf16, K-major 128B swizzle): row m of sub-chunk `part` (64 keys = 128 bytes)
+          uint8_t* pbase = smem + kOffP + part * kQChunkBytes;
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            uint8_t* dstp = pbase + (c >> 3) * kQChunkBytes + sw128_offset((uint32_t)m, (uint32_t)(c & 7));
+          for (int c = 0; c < 8; ++c) {
+            uint8_t* dstp = pbase + sw128_offset((uint32_t)m, (uint32_t)c);
             *reinterpret_cast<uint4*>(dstp) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
           }
           fence_proxy_async_smem();
@@ -502,38 +580,35 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
       }
       if (!ok) break;
       // ---- epilogue: wait for the last PV, normalise, store ----
-      ok = mbar_wait_bounded<true>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
+      ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
       pv_done_phase ^= 1;
       if (!ok) break;
       tc_fence_after_sync();
-      float l_other;
-      ok = pair_exchange(xbuf, kh, m, ++xseq, l_run, l_other, limit, abort_flag, p.status, w);
+      float l_tot = l_run;
+      ok = quad_exchange_sum(xbuf, part, m, ++xseq, l_run, l_tot, limit, abort_flag, p.status, w);
       if (!ok) break;
-      const float l_tot = l_run + l_other;
       const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
       __nv_bfloat16* Orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)(valid ? r : 0) * kDLatent;
 #pragma unroll 1
-      for (int h = 0; h < 2; ++h) {
-#pragma unroll 1
-        for (int cc = 0; cc < 128; cc += 32) {
-          uint32_t o[32];
-          tmem_ld_x32(tmem_base + lane_base + kColO + h * 128 + cc, o);
-          tmem_wait_ld();
-          if (valid) {
-            uint4* dstg = reinterpret_cast<uint4*>(Orow + 256 * h + 128 * kh + cc);
+      for (int cc = 0; cc < 128; cc += 32) {
+        const int h = cc >> 6, c0 = cc & 63;
+        uint32_t o[32];
+        tmem_ld_x32(tmem_base + lane_base + kColO + (uint32_t)(h * 128 + ch * 64 + c0), o);
+        tmem_wait_ld();
+        if (valid) {
+          uint4* dstg = reinterpret_cast<uint4*>(Orow + 256 * h + 128 * kh + 64 * ch + c0);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              uint4 v;
-              v.x = pack_bf16(__uint_as_float(o[8 * e + 0]) * inv, __uint_as_float(o[8 * e + 1]) * inv);
-              v.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
-              v.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
-              v.w = pack_bf16(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv);
-              dstg[e] = v;
-            }
+          for (int e = 0; e < 4; ++e) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(o[8 * e + 0]) * inv, __uint_as_float(o[8 * e + 1]) * inv);
+            v.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
+            v.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
+            v.w = pack_bf16(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv);
+            dstg[e] = v;
           }
         }
       }
-      if (valid && kh == 0)
+      if (valid && part == 0)
         p.lse[r] = (l_tot > 0.f) ? (m_run + log2f(l_tot)) * 0.69314718055994530942f : -INFINITY;
       tc_fence_before_sync();
     }
@@ -551,6 +626,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(256, 1)
   }
 }
 
+int g_attn_debug = 0;
+
 cudaError_t attention_setup() {
   return cudaFuncSetAttribute(rk_mla_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
 }
@@ -558,7 +635,7 @@ cudaError_t attention_setup() {
 int attention_max_pairs(int sm_count) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * (sm_count / 2), 1, 1);
-  cfg.blockDim = dim3(256, 1, 1);
+  cfg.blockDim = dim3(kAttnThreads, 1, 1);
   cfg.dynamicSmemBytes = kSmemBytes;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -576,7 +653,7 @@ int attention_max_pairs(int sm_count) {
 }
 
 cudaError_t launch_attention(const AttnParams& p, int n_pairs, cudaStream_t stream) {
-  rk_mla_attn_kernel<<<dim3(2 * n_pairs, 1, 1), dim3(256, 1, 1), kSmemBytes, stream>>>(p);
+  rk_mla_attn_kernel<<<dim3(2 * n_pairs, 1, 1), dim3(kAttnThreads, 1, 1), kSmemBytes, stream>>>(p);
   return cudaGetLastError();
 }
 

@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -199,6 +200,7 @@ rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
     return RK_ERR_CUDA;
   }
   ctx->encode = reinterpret_cast<PFN_encodeTiled>(fn);
+  if (const char* dbg = getenv("RK_ATTN_DEBUG")) g_attn_debug = atoi(dbg);
   e = attention_setup();
   if (e == cudaSuccess) e = gemm_setup();
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->d_status), sizeof(DeviceStatus));
@@ -481,6 +483,7 @@ static rk_status attn_pass(rk_ctx* ctx, const rk_request* rq, const void* kv, co
   const int n_pairs = std::min(ctx->n_pairs, n_tiles);
   p.n_pairs = n_pairs;
   p.scale_log2 = ctx->prof.sm_scale * 1.44269504088896340736f;
+  p.debug = g_attn_debug;
   cudaError_t e = launch_attention(p, n_pairs, stream);
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "attention launch");
 }

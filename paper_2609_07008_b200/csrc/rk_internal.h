@@ -43,11 +43,13 @@ struct AttnParams {
   int32_t hpt;     // heads per token in this pass (G or L)
   int32_t n_pairs;
   float scale_log2;  // sm_scale * log2(e)
+  int32_t debug;     // development switches (0 in production)
 };
 
 cudaError_t launch_attention(const AttnParams& p, int n_pairs, cudaStream_t stream);
 cudaError_t attention_setup();  // sets the dynamic shared memory attribute once
 int attention_max_pairs(int sm_count);
+extern int g_attn_debug;
 
 // ---- batched GEMM  C[M,N] = A[M,K] * B[N,K]^T  (bf16 in, fp32 accumulate, bf16 out) ----------
 struct GemmBatch {
