@@ -162,6 +162,24 @@ rk_status rk_group_sliced_proj(rk_ctx* ctx, const rk_request* req, const void* O
                                const void* W_uv, const void* W_a, void* z_on_g, void* z_on_l, void* workspace,
                                size_t workspace_bytes, void* stream);
 
+/* The same projection for callers that cannot allocate device memory (the paper has no
+ * counterpart; it is a property of this library's interface only).  A serving process that has
+ * given the whole device to its own memory pool, or a request path that must not pay the
+ * device-wide synchronisation an allocation can trigger, has no workspace to pass to
+ * rk_group_sliced_proj.  Here the per-head intermediate lives in a fixed 32 MiB
+ * (33 554 432 bytes) array inside the loaded library image; every device that loads the library
+ * holds that array until the process exits.  The call allocates and frees nothing.
+ *  - Requests whose scratch need (rk_workspace_bytes) exceeds 32 MiB are rejected with
+ *    RK_ERR_WORKSPACE and a message; use rk_group_sliced_proj with your own workspace then.
+ *  - The first call on each device looks up the array's device address (the context's device
+ *    must be current); make that first call before starting any stream capture.
+ *  - All calls, from all contexts and streams of a process, share the one array, and it keeps
+ *    whatever the previous call left in it.  Nothing in it needs to start at zero.  Two calls
+ *    whose kernels overlap on the GPU (different streams) race on it: serialise them.
+ * Arguments and results are exactly those of rk_group_sliced_proj, minus the workspace. */
+rk_status rk_group_sliced_proj_static(rk_ctx* ctx, const rk_request* req, const void* O_g, const void* O_l,
+                                      const void* W_uv, const void* W_a, void* z_on_g, void* z_on_l, void* stream);
+
 /* (5) Add the offline MLA-Off artifact and run the shared second projection (Algorithm 2:
  * RestoreAndReplace, then W_b z; "replaced, never double counted"):
  *   z[t] = z_on_g[t] + (t in A ? z_on_l[slot(t)] : z_off[t]);  y = W_b z.

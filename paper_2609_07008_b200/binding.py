@@ -47,7 +47,8 @@ class rk_layer_buffers(C.Structure):
 EXPORTS = ["rk_version", "rk_status_string", "rk_create", "rk_destroy", "rk_last_error", "rk_poll_status",
            "rk_set_wait_limit_ms", "rk_request_create", "rk_request_destroy", "rk_check_request",
            "rk_request_get_info", "rk_workspace_bytes", "rk_relocate_q", "rk_mla_online_attn",
-           "rk_segmented_merge", "rk_group_sliced_proj", "rk_combine_offline", "rk_layer_host"]
+           "rk_segmented_merge", "rk_group_sliced_proj", "rk_group_sliced_proj_static", "rk_combine_offline",
+           "rk_layer_host"]
 
 
 def _load() -> C.CDLL:
@@ -75,6 +76,7 @@ def _load() -> C.CDLL:
     lib.rk_mla_online_attn.argtypes = [vp] * 10
     lib.rk_segmented_merge.argtypes = [vp, i32, i64, i32, vp, i32, vp, vp, vp, vp]
     lib.rk_group_sliced_proj.argtypes = [vp] * 9 + [C.c_size_t, vp]
+    lib.rk_group_sliced_proj_static.argtypes = [vp] * 9
     lib.rk_combine_offline.argtypes = [vp] * 9
     lib.rk_layer_host.argtypes = [vp] * 9 + [C.POINTER(rk_layer_buffers), vp, vp]
     for name in EXPORTS:
@@ -215,6 +217,13 @@ class Context:
         self.check(lib.rk_group_sliced_proj(self.handle, req.handle, _ptr(O_g), _ptr(O_l), _ptr(W_uv), _ptr(W_a),
                                             _ptr(z_on_g), _ptr(z_on_l), _ptr(workspace), workspace.numel(),
                                             _stream()))
+        return z_on_g, z_on_l
+
+    def rk_group_sliced_proj_static(self, req, O_g, O_l, W_uv, W_a, z_on_g, z_on_l):
+        """Projection for callers that cannot allocate: outputs are passed in, the intermediate
+        lives in the library's built-in 32 MiB array (shared by all calls; see include/rk.h)."""
+        self.check(lib.rk_group_sliced_proj_static(self.handle, req.handle, _ptr(O_g), _ptr(O_l), _ptr(W_uv),
+                                                   _ptr(W_a), _ptr(z_on_g), _ptr(z_on_l), _stream()))
         return z_on_g, z_on_l
 
     def rk_combine_offline(self, req, z_on_g, z_on_l, z_off, W_b, z=None, y=None):

@@ -631,3 +631,60 @@ rk_status rk_layer_host(rk_ctx* ctx, const rk_request* rq, const void* kv_host, 
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Projection without any allocation by the caller or the library.
+//
+// Some users of this library cannot obtain device memory at call time: a serving runtime that
+// hands the whole device to its own memory pool at start-up has nothing left for cudaMalloc,
+// and a latency-critical request path cannot afford the implicit device-wide synchronisation
+// an allocation may cause.  For them the per-head intermediate o = W_uv O_lat lives in a
+// fixed array that is part of the loaded library image instead of a caller workspace.
+// ------------------------------------------------------------------------------------------
+#define RK_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+
+static __device__ __align__(256) unsigned char rk_static_scratch[RK_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_ptr[kMaxDevices] = {nullptr};
+
+// Device address of rk_static_scratch on the CURRENT device (resolved once per device).  In host
+// code the array's name is only a handle for the runtime, not a device address, so the address
+// must come from cudaGetSymbolAddress.
+cudaError_t static_scratch_address(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (g_static_scratch_ptr[device] == nullptr) {
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, rk_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_scratch_ptr[device] = ptr;
+  }
+  *out = g_static_scratch_ptr[device];
+  return cudaSuccess;
+}
+}  // namespace
+
+extern "C" rk_status rk_group_sliced_proj_static(rk_ctx* ctx, const rk_request* rq, const void* O_g, const void* O_l,
+                                                 const void* W_uv, const void* W_a, void* z_on_g, void* z_on_l,
+                                                 void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!rq) return fail(ctx, RK_ERR_NULL, "null argument");
+  if (rq->ctx != ctx) return fail(ctx, RK_ERR_LAYOUT, "request belongs to another context");
+  const size_t need = proj_ws_bytes(rq);
+  if (need > (size_t)RK_STATIC_SCRATCH_BYTES)
+    return fail(ctx, RK_ERR_WORKSPACE,
+                "request needs %zu bytes of projection scratch but the built-in array holds %u; use "
+                "rk_group_sliced_proj with a caller workspace",
+                need, (unsigned)RK_STATIC_SCRATCH_BYTES);
+  int device = -1;
+  cudaError_t e = cudaGetDevice(&device);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaGetDevice");
+  if (device != ctx->device) return fail(ctx, RK_ERR_CUDA, "the context's device is not current");
+  void* scratch = nullptr;
+  e = static_scratch_address(device, &scratch);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaGetSymbolAddress(rk_static_scratch)");
+  // nothing in the scratch has to start at zero: o is fully written before it is read, and rows
+  // beyond the tensor's extent are zero-filled by the TMA load, never read from the array
+  return rk_group_sliced_proj(ctx, rq, O_g, O_l, W_uv, W_a, z_on_g, z_on_l, scratch, RK_STATIC_SCRATCH_BYTES, stream);
+}
