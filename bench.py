@@ -28,6 +28,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 from paper_2609_07008_b200 import synth  # noqa: E402
+from paper_2609_07008_b200 import dist as rkdist  # noqa: E402
 
 FLOP_PER_PAIR = 2 * 576 + 2 * 512     # QK^T over 576 + PV over 512 per visible (row, key, head)
 L2_BYTES = 126 * 1024 * 1024
@@ -187,24 +188,20 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rk" else args.warmup
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local_rank = rkdist.env_ranks()
     if args.impl == "reference":
         run_reference(args, rank, world)
         return
 
-    import torch.distributed as dist
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    rkdist.init("nccl", dev)
     from paper_2609_07008_b200 import binding as rk   # raises if librk.so is missing: no fallback
 
     name = args.config
     prof, lay, prot = synth.make_geometry(name)
     # every rank gets its own request values (independent requests, same shape)
-    w = synth.make_tensors(name, prof, lay, prot, synth.CONFIGS[name]["seed"] * 1000 + rank, device=dev,
+    w = synth.make_tensors(name, prof, lay, prot, rkdist.rank_seed(synth.CONFIGS[name]["seed"], rank), device=dev,
                            regime=args.regime)
     ctx = rk.Context.from_profile(prof)
     req = ctx.rk_request_create(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, prot)
@@ -237,13 +234,13 @@ def main():
     sampler = ClockSampler(local_rank)
     sampler.start()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    if world > 1: dist.barrier()
+    rkdist.barrier()
     torch.cuda.synchronize()
     for i in range(args.steps):
         step(evs[i])
         if need_flush: flush_buf.fill_(1)
     torch.cuda.synchronize()
-    if world > 1: dist.barrier()
+    rkdist.barrier()
     sampler.stop_flag = True
     ctx.rk_poll_status()
     step_ms = [evs[i][0].elapsed_time(evs[i][3]) for i in range(args.steps)]
@@ -251,9 +248,7 @@ def main():
     attn_g_ms = [evs[i][0].elapsed_time(evs[i][1]) for i in range(args.steps)]
     rest_ms = [evs[i][2].elapsed_time(evs[i][3]) for i in range(args.steps)]
     total_ms = float(sum(step_ms))
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1: dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms_max = float(t.item())
+    total_ms_max = rkdist.max_over_ranks(total_ms, dev)
     sampler.join(timeout=2)
     clocks = sampler.summary()
 
@@ -264,23 +259,22 @@ def main():
         hk, hqg, hql, hzo = pin(w.kv), pin(w.q_g), pin(w.q_l), pin(w.z_off)
         y_h = torch.empty((req.T, prof.d_model), dtype=torch.bfloat16).pin_memory()
         ctx.rk_layer_host(req, hk, hqg, hql, hzo, w.w_uv, w.w_a, w.w_b, bufs, y_h)   # warm-up
-        if world > 1: dist.barrier()
+        rkdist.barrier()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         for _ in range(args.e2e_steps):
             ctx.rk_layer_host(req, hk, hqg, hql, hzo, w.w_uv, w.w_a, w.w_b, bufs, y_h)
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0)
-        te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        if world > 1: dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e_max = rkdist.max_over_ranks(e2e_s, dev)
         ctx.rk_poll_status()
-        e2e = dict(value=world * req.T * args.e2e_steps / float(te.item()), unit="tokens/s",
+        e2e = dict(value=rkdist.aggregate_throughput(req.T, args.e2e_steps, world, e2e_max), unit="tokens/s",
                    h2d_bytes_per_step=int(in_bytes), d2h_bytes_per_step=int(y_h.numel() * 2),
-                   ms_per_step=float(te.item()) * 1e3 / args.e2e_steps)
+                   ms_per_step=e2e_max * 1e3 / args.e2e_steps)
         del hk, hqg, hql, hzo
 
     if rank != 0:
-        if world > 1: dist.destroy_process_group()
+        rkdist.shutdown()
         return
 
     peaks = load_peaks()
@@ -307,7 +301,8 @@ def main():
                                    f"{dt:.1f} s, extrapolated by pair count",
                             pairs_per_s=pairs / dt, parity_rel_l2_y=rel_l2(y_gpu, out["y"]))
 
-    line = dict(metric="mla_online_prefill_tokens_per_s_per_layer", value=world * req.T * args.steps / (total_ms_max * 1e-3),
+    line = dict(metric="mla_online_prefill_tokens_per_s_per_layer",
+                value=rkdist.aggregate_throughput(req.T, args.steps, world, total_ms_max * 1e-3),
                 unit="tokens/s", n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=total_ms_max / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="bf16", data="synthetic",
@@ -318,7 +313,7 @@ def main():
                 clocks=clocks, e2e=e2e, gpu_launches=launches_per_step * args.steps, roofline=roofline,
                 proj_tflops=rest_tflops, proj_ms_per_step=float(np.mean(rest_ms)), cpu_baseline=cpu_baseline)
     print(json.dumps(line))
-    if world > 1: dist.destroy_process_group()
+    rkdist.shutdown()
 
 
 if __name__ == "__main__":
