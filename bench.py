@@ -172,6 +172,48 @@ def run_reference(args, rank, world):
 
 # ------------------------------------------------------------------------------------------------
 
+def time_stream_kernels(ctx, req, w, prof, lay, dev, budget_bytes=6 << 30):
+    """rk_relocate_q over (rows x Global heads x frames) and rk_segmented_merge over
+    (query-suffix rows x all heads x parts), each sized to a few GB, timed with CUDA events
+    after three warm-ups; algorithmic bytes = every tensor read or written once."""
+    res = {}
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, reps=5):
+        for _ in range(3):
+            fn()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, b in evs:
+            a.record(stream)
+            fn()
+            b.record(stream)
+        torch.cuda.synchronize()
+        return float(np.mean([a.elapsed_time(b) for a, b in evs]))
+
+    G, S, T = prof.n_groups, lay.n_segs, lay.n_rows
+    frame_bytes = T * G * 64 * 2
+    frames = int(max(1, min(S, budget_bytes // frame_bytes)))
+    out = torch.empty((frames, T, G, 64), dtype=torch.bfloat16, device=dev)
+    view = w.q_g[:, :, 512:]
+    ms = timed(lambda: ctx.rk_relocate_q(req, view, 0, frames, out))
+    nbytes = frame_bytes * (1 + frames)
+    res["rk_relocate_q"] = dict(ms=ms, bytes=nbytes, gbs=nbytes / ms / 1e6, frames=frames, rows=T, heads=G)
+    del out
+    H = prof.n_heads
+    n_q = int(lay.seg_off[-1] - lay.seg_off[-2])
+    part_bytes = n_q * H * (512 * 2 + 4)
+    parts = int(max(2, min(S, budget_bytes // part_bytes)))
+    O_part = torch.randn((parts, n_q, H, 512), device=dev, dtype=torch.float32).to(torch.bfloat16)
+    lse_part = torch.randn((parts, n_q, H), device=dev, dtype=torch.float32)
+    O = torch.empty((n_q, H, 512), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((n_q, H), dtype=torch.float32, device=dev)
+    ms = timed(lambda: ctx.rk_segmented_merge(O_part, lse_part, O, lse))
+    nbytes = part_bytes * parts + n_q * H * (512 * 2 + 4)
+    res["rk_segmented_merge"] = dict(ms=ms, bytes=nbytes, gbs=nbytes / ms / 1e6, parts=parts, rows=n_q, heads=H)
+    ctx.rk_poll_status()
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -185,6 +227,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-aux", action="store_true", help="skip the standalone relocation / merge timings")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rk" else args.warmup
 
@@ -204,6 +247,8 @@ def main():
     w = synth.make_tensors(name, prof, lay, prot, rkdist.rank_seed(synth.CONFIGS[name]["seed"], rank), device=dev,
                            regime=args.regime)
     ctx = rk.Context.from_profile(prof)
+    if os.environ.get("RK_DEBUG_FLAGS"):      # timing experiments only; results are meaningless then
+        ctx.rk_set_debug_flags(int(os.environ["RK_DEBUG_FLAGS"]))
     req = ctx.rk_request_create(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, prot)
     bufs = ctx.alloc_layer_buffers(req, dev)
     fl_attn, fl_proj, fl_wb = algorithmic_flops(prof, req)
@@ -273,6 +318,11 @@ def main():
                    ms_per_step=e2e_max * 1e3 / args.e2e_steps)
         del hk, hqg, hql, hzo
 
+    # standalone HBM-bound calls (not part of the step): relocation and merge against copy bandwidth
+    aux = None
+    if not args.no_aux and rank == 0:
+        aux = time_stream_kernels(ctx, req, w, prof, lay, dev)
+
     if rank != 0:
         rkdist.shutdown()
         return
@@ -312,6 +362,10 @@ def main():
                             flops_attn=fl_attn, flops_proj=fl_proj + fl_wb),
                 clocks=clocks, e2e=e2e, gpu_launches=launches_per_step * args.steps, roofline=roofline,
                 proj_tflops=rest_tflops, proj_ms_per_step=float(np.mean(rest_ms)), cpu_baseline=cpu_baseline)
+    if aux:
+        for k, v in aux.items():
+            v["frac_of_hbm_peak"] = v["gbs"] / peaks["hbm_gbs"]
+        line["hbm_kernels"] = dict(peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"] + " copy bandwidth", **aux)
     print(json.dumps(line))
     rkdist.shutdown()
 

@@ -45,7 +45,7 @@ class rk_layer_buffers(C.Structure):
 
 
 EXPORTS = ["rk_version", "rk_status_string", "rk_create", "rk_destroy", "rk_last_error", "rk_poll_status",
-           "rk_set_wait_limit_ms", "rk_request_create", "rk_request_destroy", "rk_check_request",
+           "rk_set_wait_limit_ms", "rk_set_debug_flags", "rk_request_create", "rk_request_destroy", "rk_check_request",
            "rk_request_get_info", "rk_workspace_bytes", "rk_relocate_q", "rk_mla_online_attn",
            "rk_segmented_merge", "rk_group_sliced_proj", "rk_group_sliced_proj_static", "rk_combine_offline",
            "rk_layer_host"]
@@ -67,6 +67,7 @@ def _load() -> C.CDLL:
     lib.rk_destroy.argtypes = [vp]
     lib.rk_poll_status.argtypes = [vp, vp]
     lib.rk_set_wait_limit_ms.argtypes = [vp, i32]
+    lib.rk_set_debug_flags.argtypes = [vp, i32]
     lib.rk_request_create.argtypes = [vp, C.POINTER(rk_layout), C.POINTER(i32), i64, C.POINTER(vp)]
     lib.rk_request_destroy.argtypes = [vp]
     lib.rk_check_request.argtypes = [C.POINTER(rk_layout), C.POINTER(i32), i64, C.c_char_p, C.c_size_t]
@@ -164,6 +165,9 @@ class Context:
 
     def rk_set_wait_limit_ms(self, ms: int):
         self.check(lib.rk_set_wait_limit_ms(self.handle, ms))
+
+    def rk_set_debug_flags(self, flags: int):
+        self.check(lib.rk_set_debug_flags(self.handle, flags))
 
     def rk_request_create(self, seg_off, seg_delta, seg_has_artifact, prot_rows) -> "Request":
         return Request(self, seg_off, seg_delta, seg_has_artifact, prot_rows)

@@ -206,6 +206,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
                                       W_RINGEMPTY, w))
           return false;
       }
+      if (p.debug & 8) {  // test switch: leave the stage empty so that the consumer's bounded wait expires
+        rp.advance();
+        return true;
+      }
       if (elect_one()) {
         const uint32_t full_local = bar(kBarRingFull + s);
         const uint32_t nbox = (col1 >= 0) ? 2u : 1u;
@@ -615,6 +619,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
   }
 
   // ------------------------------ teardown ---------------------------------------------------
+  // after a wait has expired: give this CTA's bulk copies that may still be in flight a bounded time
+  // to land before its shared memory goes away
+  if (*abort_flag != 0) {
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+  }
   __syncwarp();
   tc_fence_before_sync();
   __syncthreads();
@@ -625,8 +634,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     tmem_dealloc<2>(tmem_base, 512);
   }
 }
-
-int g_attn_debug = 0;
 
 cudaError_t attention_setup() {
   return cudaFuncSetAttribute(rk_mla_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);

@@ -32,6 +32,7 @@ struct rk_ctx {
   GemmBatch* d_batches = nullptr;  // [uv_g: G][uv_l: L][wa_g: G][wa_l: G][wb: 1]
   int off_uv_g = 0, off_uv_l = 0, off_wa_g = 0, off_wa_l = 0, off_wb = 0;
   unsigned long long wait_ns = 2000ull * 1000 * 1000;
+  int attn_debug = 0;  // development switches of the attention kernel (rk_set_debug_flags)
   PFN_encodeTiled encode = nullptr;
   mutable std::string err;
 };
@@ -200,7 +201,6 @@ rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
     return RK_ERR_CUDA;
   }
   ctx->encode = reinterpret_cast<PFN_encodeTiled>(fn);
-  if (const char* dbg = getenv("RK_ATTN_DEBUG")) g_attn_debug = atoi(dbg);
   e = attention_setup();
   if (e == cudaSuccess) e = gemm_setup();
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->d_status), sizeof(DeviceStatus));
@@ -257,6 +257,12 @@ rk_status rk_set_wait_limit_ms(rk_ctx* ctx, int32_t ms) {
   if (!ctx) return RK_ERR_NULL;
   if (ms <= 0) return fail(ctx, RK_ERR_PROFILE, "wait limit must be positive");
   ctx->wait_ns = (unsigned long long)ms * 1000ull * 1000ull;
+  return RK_OK;
+}
+
+rk_status rk_set_debug_flags(rk_ctx* ctx, int32_t flags) {
+  if (!ctx) return RK_ERR_NULL;
+  ctx->attn_debug = flags;
   return RK_OK;
 }
 
@@ -483,7 +489,7 @@ static rk_status attn_pass(rk_ctx* ctx, const rk_request* rq, const void* kv, co
   const int n_pairs = std::min(ctx->n_pairs, n_tiles);
   p.n_pairs = n_pairs;
   p.scale_log2 = ctx->prof.sm_scale * 1.44269504088896340736f;
-  p.debug = g_attn_debug;
+  p.debug = ctx->attn_debug;
   cudaError_t e = launch_attention(p, n_pairs, stream);
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "attention launch");
 }

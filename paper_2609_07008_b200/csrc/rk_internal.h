@@ -49,7 +49,6 @@ struct AttnParams {
 cudaError_t launch_attention(const AttnParams& p, int n_pairs, cudaStream_t stream);
 cudaError_t attention_setup();  // sets the dynamic shared memory attribute once
 int attention_max_pairs(int sm_count);
-extern int g_attn_debug;
 
 // ---- batched GEMM  C[M,N] = A[M,K] * B[N,K]^T  (bf16 in, fp32 accumulate, bf16 out) ----------
 struct GemmBatch {

@@ -227,3 +227,123 @@ def test_end_to_end_tiny_honest_artifact(rk, regime):
     ctx.rk_layer_host(req, pin(w.kv), pin(w.q_g), pin(w.q_l), pin(w.z_off), w.w_uv, w.w_a, w.w_b, bufs, y_h)
     ctx.rk_poll_status()
     assert torch.equal(y_h, y.cpu())
+
+
+# -- edge cases -------------------------------------------------------------------------------------------
+
+def _layer(rk, w):
+    ctx, req = make(rk, w)
+    to_device(w)
+    O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l if req.A else None)
+    z_on_g, z_on_l = ctx.rk_group_sliced_proj(req, O_g, O_l, w.w_uv, w.w_a)
+    z, y = ctx.rk_combine_offline(req, z_on_g, z_on_l, w.z_off if w.layout.n_doc_rows else None, w.w_b)
+    ctx.rk_poll_status()
+    return y
+
+
+def test_query_only_request(rk):
+    """No documents: one segment without artifact, every row protected, z_off never touched."""
+    w = synth.make_custom([], 37, n_heads=16, n_groups=2, o_rank=128, d_model=256, pct_bp=0, seed=41)
+    assert w.layout.n_segs == 1 and len(w.prot_rows) == 37 and w.layout.n_doc_rows == 0
+    exp = oracle_online(w, np.arange(37), z_off=np.zeros((0, 256)))
+    y = _layer(rk, w)
+    assert_close(f64(y), exp["y"], "y")
+
+
+def test_no_protected_rows(rk):
+    """Every segment has an artifact and nothing is protected: the Local pass is skipped and every row
+    takes z_off."""
+    rng = np.random.default_rng(42)
+    lay = synth.make_layout([130, 200], 0, rng, shuffle=True)
+    lay = synth.Layout(seg_off=lay.seg_off[:-1], seg_delta=lay.seg_delta[:-1], seg_has_artifact=lay.seg_has_artifact[:-1])
+    prof = synth.Profile(n_heads=16, n_groups=2, o_rank=128, d_model=256, global_heads=synth.draw_global_heads(2, rng),
+                         sm_scale=float(1 / np.sqrt(192)))
+    w = synth.make_tensors("custom", prof, lay, np.zeros(0, np.int32), 42, regime="sharp")
+    exp = oracle_online(w, np.arange(lay.n_rows))
+    y = _layer(rk, w)
+    assert_close(f64(y), exp["y"], "y")
+
+
+def test_gaps_between_segments_and_large_offsets(rk):
+    """Request-position intervals need not be contiguous: offsets with gaps (and beyond 2^20, where the
+    relocation angles are large) leave the result equal to the checker's."""
+    w = synth.make_custom([100, 260, 31], 20, n_heads=16, n_groups=2, o_rank=128, d_model=256, pct_bp=1000, seed=43)
+    lay = w.layout
+    lay.seg_delta = lay.seg_delta * 3 + np.array([7, 1 << 20, 12345, 5 << 20])[: lay.n_segs]
+    # keep intervals disjoint
+    order = np.argsort(lay.seg_delta)
+    ends = lay.seg_delta[order] + (lay.seg_off[1:] - lay.seg_off[:-1])[order]
+    assert (lay.seg_delta[order][1:] >= ends[:-1]).all()
+    exp = oracle_online(w, np.arange(lay.n_rows))
+    ctx, req = make(rk, w)
+    to_device(w)
+    O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
+    ctx.rk_poll_status()
+    assert_close(f64(O_g), exp["O_g"], "O_g")
+    assert_close(f64(O_l), exp["O_l"], "O_l")
+    assert max_abs(f64(lse_g), exp["lse_g"]) <= LSE_TOL["sharp"]
+
+
+def test_argument_errors_on_device(rk):
+    """Errors that need a context: misaligned pointers, short workspace, half-specified passes, a
+    request from another context.  All are reported before anything is enqueued."""
+    w = small_ragged(seed=12)
+    ctx, req = make(rk, w)
+    ctx2, _ = make(rk, w)
+    to_device(w)
+    T, A, p = w.layout.n_rows, len(w.prot_rows), w.profile
+    O_g = torch.empty((T, p.n_groups, 512), dtype=torch.bfloat16, device="cuda")
+    lse_g = torch.empty((T, p.n_groups), dtype=torch.float32, device="cuda")
+    L = rk.lib
+    s = torch.cuda.current_stream().cuda_stream
+    # misaligned kv (2-byte offset)
+    kv_pad = torch.empty(T * 576 + 8, dtype=torch.bfloat16, device="cuda")
+    assert L.rk_mla_online_attn(ctx.handle, req.handle, kv_pad.data_ptr() + 2, w.q_g.data_ptr(), None, O_g.data_ptr(),
+                                lse_g.data_ptr(), None, None, s) == 5
+    # Global pass half specified
+    assert L.rk_mla_online_attn(ctx.handle, req.handle, w.kv.data_ptr(), w.q_g.data_ptr(), None, None, None, None,
+                                None, s) == 1
+    # request created by another context
+    assert L.rk_mla_online_attn(ctx2.handle, req.handle, w.kv.data_ptr(), w.q_g.data_ptr(), None, O_g.data_ptr(),
+                                lse_g.data_ptr(), None, None, s) == 3
+    # workspace one byte short
+    ws = torch.empty(req.workspace_bytes, dtype=torch.uint8, device="cuda")
+    z = torch.empty((T, p.n_groups * p.o_rank), dtype=torch.bfloat16, device="cuda")
+    assert L.rk_group_sliced_proj(ctx.handle, req.handle, O_g.data_ptr(), None, w.w_uv.data_ptr(), w.w_a.data_ptr(),
+                                  z.data_ptr(), None, ws.data_ptr(), req.workspace_bytes - 1, s) == 6
+    assert b"workspace" in L.rk_last_error(ctx.handle)
+    # relocation: segment range out of bounds, stride not a multiple of 8
+    out = torch.empty((1, T, p.n_groups, 64), dtype=torch.bfloat16, device="cuda")
+    assert L.rk_relocate_q(ctx.handle, req.handle, w.q_g.data_ptr(), T, p.n_groups, 576 * p.n_groups, 576, 0,
+                           w.layout.n_segs + 1, out.data_ptr(), s) == 3
+    assert L.rk_relocate_q(ctx.handle, req.handle, w.q_g.data_ptr(), T, p.n_groups, 577 * p.n_groups, 577, 0, 1,
+                           out.data_ptr(), s) == 5
+    # merge: unknown part dtype
+    assert L.rk_segmented_merge(ctx.handle, 2, 4, 2, O_g.data_ptr(), 7, lse_g.data_ptr(), O_g.data_ptr(),
+                                lse_g.data_ptr(), s) == 7
+    # combine: W_b given without y
+    assert L.rk_combine_offline(ctx.handle, req.handle, z.data_ptr(), z.data_ptr(), z.data_ptr(), w.w_b.data_ptr(),
+                                z.data_ptr(), None, s) == 1
+    ctx.rk_poll_status()          # nothing was enqueued, nothing timed out
+
+
+def test_bounded_wait_reports_timeout_and_context_stays_usable(rk):
+    """A device-side wait that nothing satisfies (the load warp is told to leave the ring stages empty)
+    expires after the configured limit: the kernel drains and returns, rk_poll_status reports
+    RK_ERR_TIMEOUT once, and the next call on the same context works."""
+    w = synth.make_workload("tiny")
+    ctx, req = make(rk, w)
+    to_device(w)
+    ctx.rk_set_wait_limit_ms(20)
+    ctx.rk_set_debug_flags(8)
+    ctx.rk_mla_online_attn(req, w.kv, w.q_g, None)
+    with pytest.raises(rk.RKError) as ei:
+        ctx.rk_poll_status()
+    assert ei.value.status == 9 and "wait expired" in str(ei.value)
+    ctx.rk_poll_status()                                   # the status word was cleared
+    ctx.rk_set_debug_flags(0)
+    ctx.rk_set_wait_limit_ms(2000)
+    exp = oracle_online(w, np.arange(w.layout.n_rows))
+    O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
+    ctx.rk_poll_status()
+    assert_close(f64(O_g), exp["O_g"], "O_g after a timed-out launch")
