@@ -102,8 +102,8 @@ const char* rk_last_error(const rk_ctx* ctx);
 rk_status rk_poll_status(rk_ctx* ctx, void* stream);
 /* Per-wait time limit of device-side waits, in milliseconds (default 2000). */
 rk_status rk_set_wait_limit_ms(rk_ctx* ctx, int32_t ms);
-/* Development switches of the attention kernel (0 = production).  Bits 0-2 remove the softmax
- * arithmetic, the tile loads or the row-maximum exchange for timing experiments (results are then
+/* Development switches of the attention kernel (0 = production).  Bit 0 removes the softmax
+ * arithmetic and bit 2 the row-maximum exchange, for timing experiments (results are then
  * meaningless).  Bit 3 makes the load warp leave every ring stage empty, so the consumer's bounded
  * wait expires and the kernel returns with RK_ERR_TIMEOUT in the status word: the test of the
  * timeout path uses it together with a short rk_set_wait_limit_ms. */

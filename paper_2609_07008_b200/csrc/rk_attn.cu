@@ -198,6 +198,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     uint32_t qfree_phase = 0;
     bool ok = true;
     int n_done = 0;
+    const uint64_t pol_kv = l2_policy_evict_last(), pol_q = l2_policy_evict_first();
     // fills one stage with one or two boxes; every lane waits, one lane issues
     auto fill = [&](int col0, int col1, int row, int w) -> bool {
       const uint32_t s = rp.stage();
@@ -213,15 +214,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       if (elect_one()) {
         const uint32_t full_local = bar(kBarRingFull + s);
         const uint32_t nbox = (col1 >= 0) ? 2u : 1u;
-        if (p.debug & 2) {
-          if (leader) mbar_arrive(full_local);
-        } else {
-          if (leader) mbar_arrive_expect_tx(full_local, 2 * nbox * kChunkBytes);
-          const uint32_t full_remote = mapa_shared(full_local, 0);
-          const uint32_t dst = smem_base + kOffRing + s * kStageBytes;
-          tma_load_2d_pair(dst, &p.tm_kv, full_remote, col0, row);
-          if (col1 >= 0) tma_load_2d_pair(dst + kChunkBytes, &p.tm_kv, full_remote, col1, row);
-        }
+        if (leader) mbar_arrive_expect_tx(full_local, 2 * nbox * kChunkBytes);
+        const uint32_t full_remote = mapa_shared(full_local, 0);
+        const uint32_t dst = smem_base + kOffRing + s * kStageBytes;
+        tma_load_2d_pair_hint(dst, &p.tm_kv, full_remote, col0, row, pol_kv);
+        if (col1 >= 0) tma_load_2d_pair_hint(dst + kChunkBytes, &p.tm_kv, full_remote, col1, row, pol_kv);
       }
       __syncwarp();
       rp.advance();
@@ -253,7 +250,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         mbar_arrive_expect_tx(bar(kBarQFull), 9 * kQChunkBytes);
         const int qrow = item.tile * kAttnRowsPerPair + (int)crank * kAttnRowsPerCta;
         for (int d = 0; d < 9; ++d)
-          tma_load_2d(smem_base + kOffQLat + d * kQChunkBytes, &p.tm_q, bar(kBarQFull), d * 64, qrow);
+          tma_load_2d_hint(smem_base + kOffQLat + d * kQChunkBytes, &p.tm_q, bar(kBarQFull), d * 64, qrow, pol_q);
       }
       __syncwarp();
       // order of consumption: K(0), K(1), V(0), K(2), V(1), ..., V(last)
@@ -608,7 +605,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             v.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
             v.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
             v.w = pack_bf16(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv);
-            dstg[e] = v;
+            __stcs(dstg + e, v);
           }
         }
       }
