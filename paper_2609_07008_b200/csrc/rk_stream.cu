@@ -35,14 +35,17 @@ __global__ void __launch_bounds__(256) rk_relocate_kernel(const __nv_bfloat16* _
        it += (int64_t)gridDim.x * blockDim.x) {
     const int c = (int)(it & 7);
     const int64_t rh = it >> 3;
-    const int64_t r = rh / n_heads;
+    const int64_t r = (rh < (int64_t)0x7fffffff) ? (int64_t)((uint32_t)rh / (uint32_t)n_heads) : rh / n_heads;
     const int h = (int)(rh - r * n_heads);
     const uint4 v = *reinterpret_cast<const uint4*>(q + r * row_stride + h * head_stride + c * 8);
     float x[8];
     unpack8(v, x);
     __nv_bfloat16* dst = out + it * 8;
+    // Frames are whole multiples of a megabyte apart, so writing frame i from every block at the same
+    // time would hit the same memory channels; each block starts at a different frame instead.
+    int i = (int)(blockIdx.x % (unsigned)n_frames);
 #pragma unroll 4
-    for (int i = 0; i < n_frames; ++i) {
+    for (int n = 0; n < n_frames; ++n) {
       const float4* cs = reinterpret_cast<const float4*>(seg_cs + (size_t)(seg_begin + i) * 32 + 4 * c);
       const float4 t01 = __ldg(cs), t23 = __ldg(cs + 1);
       float y[8];
@@ -52,6 +55,7 @@ __global__ void __launch_bounds__(256) rk_relocate_kernel(const __nv_bfloat16* _
       y[4] = x[4] * t23.x + x[5] * t23.y;  y[5] = x[5] * t23.x - x[4] * t23.y;
       y[6] = x[6] * t23.z + x[7] * t23.w;  y[7] = x[7] * t23.z - x[6] * t23.w;
       __stcs(reinterpret_cast<uint4*>(dst + (int64_t)i * frame_elems), pack8(y));
+      i = (i + 1 == n_frames) ? 0 : i + 1;
     }
   }
 }
