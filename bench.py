@@ -214,6 +214,45 @@ def time_stream_kernels(ctx, req, w, prof, lay, dev, budget_bytes=6 << 30):
     return res
 
 
+def time_offline_build(ctx, req, w, prof, lay, dev, rows_per_call=65536):
+    """Offline MLA-Off artifact build (Algorithm 1) over every document row, in row ranges; not part of
+    the online step.  Flops: 2176 per visible (row, key, Local head) pair inside each document alone,
+    plus the Local half of the sliced projection."""
+    n, L, G, ro = lay.n_doc_rows, prof.n_local, prof.n_groups, prof.o_rank
+    rows_per_call = min(rows_per_call, n)
+    q = (torch.randn((rows_per_call, L, 576), device=dev, dtype=torch.float32)).to(torch.bfloat16)
+    z = torch.empty((rows_per_call, G * ro), dtype=torch.bfloat16, device=dev)
+    import ctypes as C
+    from paper_2609_07008_b200 import binding as rk
+    ws_n = C.c_size_t()
+    rk.lib.rk_mla_off_workspace_bytes(req.handle, rows_per_call, C.byref(ws_n))
+    ws = torch.empty(ws_n.value, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    pairs = 0
+    for i in range(lay.n_segs):
+        if lay.seg_has_artifact[i]:
+            m = int(lay.seg_off[i + 1] - lay.seg_off[i])
+            pairs += m * (m + 1) // 2
+    flops = 2176 * L * pairs + 2 * n * (L * 512 * 128 + G * 7 * 128 * ro)
+
+    def run():
+        for lo in range(0, n, rows_per_call):
+            hi = min(n, lo + rows_per_call)
+            ctx.rk_mla_off_build(req, w.kv, lo, hi, q[: hi - lo], w.w_uv, w.w_a, z[: hi - lo], ws)
+
+    run()
+    run()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    run()
+    b.record(stream)
+    torch.cuda.synchronize()
+    ctx.rk_poll_status()
+    ms = a.elapsed_time(b)
+    return dict(ms=ms, rows=n, tokens_per_s=n / ms * 1e3, tflops=flops / ms / 1e9, rows_per_call=rows_per_call,
+                flops=flops)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -228,6 +267,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-aux", action="store_true", help="skip the standalone relocation / merge timings")
+    ap.add_argument("--with-offline", action="store_true", help="also time the offline artifact build")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rk" else args.warmup
 
@@ -323,6 +363,10 @@ def main():
     if not args.no_aux and rank == 0:
         aux = time_stream_kernels(ctx, req, w, prof, lay, dev)
 
+    offline = None
+    if args.with_offline and rank == 0:
+        offline = time_offline_build(ctx, req, w, prof, lay, dev)
+
     if rank != 0:
         rkdist.shutdown()
         return
@@ -362,6 +406,8 @@ def main():
                             flops_attn=fl_attn, flops_proj=fl_proj + fl_wb),
                 clocks=clocks, e2e=e2e, gpu_launches=launches_per_step * args.steps, roofline=roofline,
                 proj_tflops=rest_tflops, proj_ms_per_step=float(np.mean(rest_ms)), cpu_baseline=cpu_baseline)
+    if offline:
+        line["offline_build"] = offline
     if aux:
         for k, v in aux.items():
             v["frac_of_hbm_peak"] = v["gbs"] / peaks["hbm_gbs"]

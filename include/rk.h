@@ -195,6 +195,22 @@ rk_status rk_group_sliced_proj_static(rk_ctx* ctx, const rk_request* req, const 
 rk_status rk_combine_offline(rk_ctx* ctx, const rk_request* req, const void* z_on_g, const void* z_on_l,
                              const void* z_off, const void* W_b, void* z, void* y, void* stream);
 
+/* Offline side (Algorithm 1 "Build one canonical MLA-Off document artifact"): for packed rows
+ * [row_begin, row_end) each row attends only the keys of its own segment, causally in the
+ * segment's position-zero frame, with the Local heads; then z_off = W_{a,L} (W_uv O_L) summed over
+ * each group's seven Local heads.  Queries are given at their REQUEST positions (like q_l); the
+ * kernel rotates them by -seg_delta into the document's frame, which is the query the document had
+ * when it was processed alone at position zero.
+ *   q_l_rows   device bf16 [row_end-row_begin][L][576]
+ *   z_off_rows device bf16 [row_end-row_begin][G*r_o]  (row row_begin of the artifact tensor)
+ *   workspace  device scratch of at least rk_mla_off_workspace_bytes(req, row_end-row_begin)
+ * Long requests are built in several calls over row ranges (the scratch holds the Local-head
+ * attention output of the range). */
+rk_status rk_mla_off_workspace_bytes(const rk_request* req, int64_t n_rows, size_t* out);
+rk_status rk_mla_off_build(rk_ctx* ctx, const rk_request* req, const void* kv, int64_t row_begin, int64_t row_end,
+                           const void* q_l_rows, const void* W_uv, const void* W_a, void* z_off_rows, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
 /* Device buffers that rk_layer_host stages through; all owned by the caller. */
 typedef struct rk_layer_buffers {
   void *kv, *q_g, *q_l, *z_off;            /* device copies of the per-request inputs */

@@ -285,20 +285,22 @@ def full_recompute_rows(rows: np.ndarray, q_all_rows: np.ndarray, kv: np.ndarray
 
 def mla_off_artifact(seg: int, q_local_doc: np.ndarray, kv: np.ndarray, seg_off, seg_delta,
                      local_heads: np.ndarray, w_uv: np.ndarray, w_a: np.ndarray, sm_scale: float,
-                     base: float, d_latent: int, group_size: int = 8) -> np.ndarray:
+                     base: float, d_latent: int, group_size: int = 8, rows: np.ndarray | None = None) -> np.ndarray:
     """Algorithm 1 for one document: the document alone at positions 0..n-1, causal over its
     own keys only, Local heads only, z_off = W_{a,L} O_L.  q_local_doc [n, L, d_qk] are the
     request-position queries of the document's rows; the query the document had at
-    position zero is R(-delta_i) of that.  Returns [n, G*r_o]."""
+    position zero is R(-delta_i) of that.  Returns [n, G*r_o].  With `rows` (canonical indices
+    inside the document) only those rows are evaluated and q_local_doc holds just their queries."""
     lo, hi = int(seg_off[seg]), int(seg_off[seg + 1])
     n = hi - lo
     q0 = np.asarray(q_local_doc, dtype=np.float64).copy()
     q0[..., d_latent:] = relocate_query(q0[..., d_latent:], float(seg_delta[seg]), base)
     kd = np.asarray(kv, dtype=np.float64)[lo:hi]
     canon = np.arange(n, dtype=np.int64)
-    O, _ = attend_rows(q0, canon, kd, kd[:, :d_latent], canon, sm_scale)
+    row_canon = canon if rows is None else np.asarray(rows, dtype=np.int64)
+    O, _ = attend_rows(q0, row_canon, kd, kd[:, :d_latent], canon, sm_scale)
     c = head_contributions(O, local_heads, w_uv, w_a, group_size)
-    return _group_sum(c, local_heads, w_a.shape[0], group_size).reshape(n, -1)
+    return _group_sum(c, local_heads, w_a.shape[0], group_size).reshape(len(row_canon), -1)
 
 
 # ---------------------------------------------------------------------------------

@@ -48,7 +48,7 @@ EXPORTS = ["rk_version", "rk_status_string", "rk_create", "rk_destroy", "rk_last
            "rk_set_wait_limit_ms", "rk_set_debug_flags", "rk_request_create", "rk_request_destroy", "rk_check_request",
            "rk_request_get_info", "rk_workspace_bytes", "rk_relocate_q", "rk_mla_online_attn",
            "rk_segmented_merge", "rk_group_sliced_proj", "rk_group_sliced_proj_static", "rk_combine_offline",
-           "rk_layer_host"]
+           "rk_layer_host", "rk_mla_off_workspace_bytes", "rk_mla_off_build"]
 
 
 def _load() -> C.CDLL:
@@ -80,6 +80,8 @@ def _load() -> C.CDLL:
     lib.rk_group_sliced_proj_static.argtypes = [vp] * 9
     lib.rk_combine_offline.argtypes = [vp] * 9
     lib.rk_layer_host.argtypes = [vp] * 9 + [C.POINTER(rk_layer_buffers), vp, vp]
+    lib.rk_mla_off_workspace_bytes.argtypes = [vp, i64, C.POINTER(C.c_size_t)]
+    lib.rk_mla_off_build.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp, vp, vp, C.c_size_t, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is C.c_int:  # default restype: rk_status
@@ -239,6 +241,20 @@ class Context:
         self.check(lib.rk_combine_offline(self.handle, req.handle, _ptr(z_on_g), _ptr(z_on_l), _ptr(z_off),
                                           _ptr(W_b), _ptr(z), _ptr(y), _stream()))
         return z, y
+
+    def rk_mla_off_build(self, req, kv, row_begin, row_end, q_l_rows, W_uv, W_a, z_off_rows=None, workspace=None):
+        """Offline artifact rows [row_begin, row_end): documents alone at position zero, Local heads."""
+        n = row_end - row_begin
+        if z_off_rows is None:
+            z_off_rows = torch.empty((n, self.n_groups * self.o_rank), dtype=torch.bfloat16, device=kv.device)
+        ws = C.c_size_t()
+        self.check(lib.rk_mla_off_workspace_bytes(req.handle, n, C.byref(ws)))
+        if workspace is None:
+            workspace = torch.empty(max(ws.value, 256), dtype=torch.uint8, device=kv.device)
+        self.check(lib.rk_mla_off_build(self.handle, req.handle, _ptr(kv), row_begin, row_end, _ptr(q_l_rows),
+                                        _ptr(W_uv), _ptr(W_a), _ptr(z_off_rows), _ptr(workspace), workspace.numel(),
+                                        _stream()))
+        return z_off_rows
 
     def alloc_layer_buffers(self, req, device) -> dict:
         G, L, T, A = self.n_groups, self.n_local, req.T, req.A

@@ -58,22 +58,44 @@ constexpr uint32_t kIdescPV = umma_idesc_bf16(128, 256, 0, 1);
 enum { W_QFULL = 1, W_QFREE, W_QRREADY, W_QRFREE, W_RINGFULL, W_RINGEMPTY, W_SFULL, W_PREADY, W_PVDONE, W_DRAIN };
 
 struct SegIter {
-  // iterates the segments a row tile can see; kmax = number of canonical keys any row may see
+  // Iterates the segments a row tile can see; kmax = number of canonical keys of the segment that
+  // any row of the tile may see.  Online mode: everything at request positions <= the tile's
+  // largest position.  Isolated mode (offline artifact build): only the segments the tile's own
+  // packed rows [prow0, prow1] lie in, each up to the tile's last row in it.
   const AttnParams& p;
-  int maxpos;
+  int maxpos, prow0, prow1;
   int seg;
   int kmax;
-  __device__ SegIter(const AttnParams& p_, int maxpos_) : p(p_), maxpos(maxpos_), seg(-1), kmax(0) {}
+  __device__ SegIter(const AttnParams& p_, const AttnWorkItem& item) : p(p_), maxpos(item.maxpos), seg(-1), kmax(0) {
+    const int r0 = item.tile * kAttnRowsPerPair;
+    int r1 = r0 + kAttnRowsPerPair - 1;
+    if (r1 > p.n_flat - 1) r1 = p.n_flat - 1;
+    prow0 = p.row_base + r0 / p.hpt;
+    prow1 = p.row_base + r1 / p.hpt;
+  }
   __device__ bool next() {
     while (++seg < p.n_segs) {
-      int n = p.seg_off[seg + 1] - p.seg_off[seg];
-      int lim = maxpos - p.seg_delta[seg] + 1;
-      kmax = lim < n ? lim : n;
+      const int lo = p.seg_off[seg], hi = p.seg_off[seg + 1];
+      if (p.isolated) {
+        if (prow1 < lo || prow0 >= hi) { kmax = 0; continue; }
+        kmax = (prow1 < hi ? prow1 : hi - 1) - lo + 1;
+      } else {
+        const int lim = maxpos - p.seg_delta[seg] + 1;
+        kmax = lim < hi - lo ? lim : hi - lo;
+      }
       if (kmax > 0) return true;
     }
     return false;
   }
 };
+
+__device__ __forceinline__ AttnWorkItem get_work(const AttnParams& p, int w) {
+  if (p.work != nullptr) return p.work[w];
+  AttnWorkItem it;  // natural order (isolated mode has no host-built list)
+  it.tile = w;
+  it.maxpos = 0;
+  return it;
+}
 
 // Ring bookkeeping shared by the producer and the UMMA issuer: both walk the same stage
 // sequence.  A stage holds two 16 KB boxes: two 64-dim K chunks (QK^T), the single rope chunk,
@@ -87,8 +109,8 @@ struct RingPos {
 };
 
 // number of key tiles a row tile walks through (all visible segments)
-__device__ __forceinline__ int count_key_tiles(const AttnParams& p, int maxpos) {
-  SegIter it(p, maxpos);
+__device__ __forceinline__ int count_key_tiles(const AttnParams& p, const AttnWorkItem& item) {
+  SegIter it(p, item);
   int n = 0;
   while (it.next()) n += (it.kmax + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
   return n;
@@ -239,7 +261,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       return true;
     };
     for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs, ++n_done) {
-      const AttnWorkItem item = p.work[w];
+      const AttnWorkItem item = get_work(p, w);
       // Q tile: wait until the previous tile's QK^T MMAs have finished reading it
       if (n_done > 0) {
         ok = mbar_wait_bounded<false>(bar(kBarQFree), qfree_phase, limit, abort_flag, p.status, W_QFREE, w);
@@ -254,7 +276,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       }
       __syncwarp();
       // order of consumption: K(0), K(1), V(0), K(2), V(1), ..., V(last)
-      SegIter it(p, item.maxpos);
+      SegIter it(p, item);
       int prev_row0 = -1, prev_kb = 0;
       while (ok && it.next()) {
         const int row0 = p.seg_off[it.seg];
@@ -290,8 +312,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       const uint32_t p_base = smem_base + kOffP;
 
       for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
-        const AttnWorkItem item = p.work[w];
-        const int n_kt = count_key_tiles(p, item.maxpos);
+        const AttnWorkItem item = get_work(p, w);
+        const int n_kt = count_key_tiles(p, item);
         int kt_issued = 0;  // key tiles whose QK^T has been issued
         int kt_pv = 0;      // key tiles whose PV has been issued
 
@@ -370,7 +392,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           return true;
         };
 
-        SegIter it(p, item.maxpos);
+        SegIter it(p, item);
         while (ok && it.next()) {
           const uint32_t rb = qr_use & 1u;
           ++qr_use;
@@ -391,10 +413,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     uint32_t qr_use = 0;
     bool ok = true;
     for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
-      const AttnWorkItem item = p.work[w];
+      const AttnWorkItem item = get_work(p, w);
       ok = mbar_wait_bounded<false>(bar(kBarQFull), qfull_phase, limit, abort_flag, p.status, W_QFULL, w);
       qfull_phase ^= 1;
-      SegIter it(p, item.maxpos);
+      SegIter it(p, item);
       while (ok && it.next()) {
         const uint32_t rb = qr_use & 1u;
         if (qr_use >= 2) {
@@ -460,24 +482,28 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     const uint32_t p_ready_remote = mapa_shared(bar(kBarPReady), 0);
 
     for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
-      const AttnWorkItem item = p.work[w];
+      const AttnWorkItem item = get_work(p, w);
       const int r = item.tile * kAttnRowsPerPair + (int)crank * kAttnRowsPerCta + m;
       const bool valid = r < p.n_flat;
-      int pos = -1;
+      int pos = -1, prow = -1;
       if (valid) {
         const int tok = r / p.hpt;
-        const int prow = p.rowmap ? p.rowmap[tok] : tok;
+        prow = p.rowmap ? p.rowmap[tok] : p.row_base + tok;
         pos = p.row_pos[prow];
       }
       float m_run = -INFINITY, l_run = 0.f;
       int kt = 0;
 
-      SegIter it(p, item.maxpos);
+      SegIter it(p, item);
       while (ok && it.next()) {
         const int n_seg = p.seg_off[it.seg + 1] - p.seg_off[it.seg];
         int lim = pos - p.seg_delta[it.seg];  // last visible canonical index
         if (lim > n_seg - 1) lim = n_seg - 1;
         if (pos < 0) lim = -1;
+        if (p.isolated) {  // only the row's own segment, causal in its canonical frame
+          const int lo = p.seg_off[it.seg];
+          lim = (prow >= lo && prow < lo + n_seg) ? prow - lo : -1;
+        }
         for (int kb = 0; kb < it.kmax && ok; kb += kAttnKeysPerTile, ++kt) {
           int nv = lim - (kb + part * 64) + 1;
           nv = nv < 0 ? 0 : (nv > 64 ? 64 : nv);

@@ -463,7 +463,7 @@ rk_status rk_relocate_q(rk_ctx* ctx, const rk_request* rq, const void* q_rope, i
 
 static rk_status attn_pass(rk_ctx* ctx, const rk_request* rq, const void* kv, const void* q, int64_t n_tok, int hpt,
                            const int32_t* rowmap, const AttnWorkItem* work, int n_tiles, void* O, float* lse,
-                           cudaStream_t stream) {
+                           cudaStream_t stream, int isolated = 0, int64_t row_base = 0) {
   if (n_tiles == 0) return RK_OK;
   AttnParams p;
   memset(&p, 0, sizeof(p));
@@ -490,6 +490,8 @@ static rk_status attn_pass(rk_ctx* ctx, const rk_request* rq, const void* kv, co
   p.n_pairs = n_pairs;
   p.scale_log2 = ctx->prof.sm_scale * 1.44269504088896340736f;
   p.debug = ctx->attn_debug;
+  p.isolated = isolated;
+  p.row_base = (int32_t)row_base;
   cudaError_t e = launch_attention(p, n_pairs, stream);
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "attention launch");
 }
@@ -512,6 +514,54 @@ rk_status rk_mla_online_attn(rk_ctx* ctx, const rk_request* rq, const void* kv, 
     s = attn_pass(ctx, rq, kv, q_l, rq->A, (int)ctx->local_heads.size(), rq->d_prot_rows, rq->d_work_l, rq->n_tiles_l,
                   O_l, lse_l, st);
   return s;
+}
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+static rk_status run_gemm(rk_ctx* ctx, const void* A, int64_t a_rows, int64_t a_cols, const void* B, int64_t b_rows,
+                          int64_t b_cols, void* C, int64_t ldc, int M, int N, int K, int batch_off, int n_batches,
+                          cudaStream_t st);
+
+rk_status rk_mla_off_workspace_bytes(const rk_request* rq, int64_t n_rows, size_t* out) {
+  if (!rq || !out) return RK_ERR_NULL;
+  if (n_rows < 0) return RK_ERR_LAYOUT;
+  const size_t L = rq->ctx->local_heads.size();
+  *out = align256((size_t)n_rows * L * kDLatent * 2) + align256((size_t)n_rows * L * 4) +
+         align256((size_t)n_rows * L * kDV * 2);
+  return RK_OK;
+}
+
+rk_status rk_mla_off_build(rk_ctx* ctx, const rk_request* rq, const void* kv, int64_t row_begin, int64_t row_end,
+                           const void* q_l_rows, const void* W_uv, const void* W_a, void* z_off_rows, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!rq || !kv || !q_l_rows || !W_uv || !W_a || !z_off_rows || !workspace) return fail(ctx, RK_ERR_NULL, "null argument");
+  if (rq->ctx != ctx) return fail(ctx, RK_ERR_LAYOUT, "request belongs to another context");
+  if (row_begin < 0 || row_end > rq->T || row_begin > row_end) return fail(ctx, RK_ERR_LAYOUT, "row range out of bounds");
+  if (!aligned16(kv) || !aligned16(q_l_rows) || !aligned16(W_uv) || !aligned16(W_a) || !aligned16(z_off_rows) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return fail(ctx, RK_ERR_ALIGN, "tensors must be 16-byte aligned and the workspace 256-byte aligned");
+  const int64_t n = row_end - row_begin;
+  size_t need = 0;
+  rk_mla_off_workspace_bytes(rq, n, &need);
+  if (workspace_bytes < need) return fail(ctx, RK_ERR_WORKSPACE, "workspace too small: need %zu bytes", need);
+  if (n == 0) return RK_OK;
+  const int G = ctx->prof.n_groups, H = ctx->prof.n_heads, L = H - G, ro = ctx->prof.o_rank;
+  if (n * L >= ((int64_t)1 << 31)) return fail(ctx, RK_ERR_LAYOUT, "row range too long for one call: split it");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  void* O = ws;
+  float* lse = reinterpret_cast<float*>(ws + align256((size_t)n * L * kDLatent * 2));
+  void* o = reinterpret_cast<uint8_t*>(lse) + align256((size_t)n * L * 4);
+  const int n_tiles = (int)((n * L + kAttnRowsPerPair - 1) / kAttnRowsPerPair);
+  // documents alone: a row sees only its own segment, causally, with the query relocated into
+  // the segment's position-zero frame; tiles in natural order (no host-built list)
+  rk_status s = attn_pass(ctx, rq, kv, q_l_rows, n, L, nullptr, nullptr, n_tiles, O, lse, st, 1, row_begin);
+  if (s != RK_OK) return s;
+  s = run_gemm(ctx, O, n, (int64_t)L * kDLatent, W_uv, (int64_t)H * kDV, kDLatent, o, (int64_t)L * kDV, (int)n, kDV,
+               kDLatent, ctx->off_uv_l, L, st);
+  if (s != RK_OK) return s;
+  return run_gemm(ctx, o, n, (int64_t)L * kDV, W_a, (int64_t)G * ro, kGroup * kDV, z_off_rows, (int64_t)G * ro, (int)n, ro,
+                  (kGroup - 1) * kDV, ctx->off_wa_l, G, st);
 }
 
 rk_status rk_segmented_merge(rk_ctx* ctx, int32_t n_parts, int64_t n_rows, int32_t n_heads, const void* O_part,

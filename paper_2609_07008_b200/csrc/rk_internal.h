@@ -44,6 +44,8 @@ struct AttnParams {
   int32_t n_pairs;
   float scale_log2;  // sm_scale * log2(e)
   int32_t debug;     // development switches (0 in production)
+  int32_t isolated;  // 1: a row sees only its own segment (documents built alone, Algorithm 1)
+  int32_t row_base;  // packed row of token slot 0 when rowmap is null
 };
 
 cudaError_t launch_attention(const AttnParams& p, int n_pairs, cudaStream_t stream);

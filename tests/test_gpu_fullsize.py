@@ -219,3 +219,29 @@ def test_document_split_gpu_vs_gpu(rk):
     ctx2.rk_poll_status()
     assert rel_l2(f64(O2), f64(O1)) <= 1e-2
     assert max_abs(f64(l2), f64(l1)) <= 1e-2
+
+
+def test_offline_artifact_build_full_size_sampled_rows(rk):
+    """rk_mla_off_build over all 32 768 document rows of the flash1 layout (built in two row ranges);
+    sampled rows of three documents against the checker's position-zero artifact."""
+    prof, lay, prot = synth.make_geometry("flash1")
+    n, L = lay.n_doc_rows, prof.n_local
+    g = torch.Generator(device="cuda").manual_seed(77)
+    kv = torch.randn((lay.n_rows, 576), generator=g, device="cuda").to(torch.bfloat16)
+    q_l_doc = (torch.randn((n, L, 576), generator=g, device="cuda") * 1.2).to(torch.bfloat16)
+    w_uv = (torch.randn((prof.n_heads, 128, 512), generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    w_a = (torch.randn((prof.n_groups, prof.o_rank, 1024), generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    ctx, req = make(rk, prof, lay, prot)
+    half = 5 * 4096 + 1234
+    z_off = torch.cat([ctx.rk_mla_off_build(req, kv, 0, half, q_l_doc[:half].contiguous(), w_uv, w_a),
+                       ctx.rk_mla_off_build(req, kv, half, n, q_l_doc[half:].contiguous(), w_uv, w_a)])
+    ctx.rk_poll_status()
+    assert torch.isfinite(z_off.float()).all()
+    kv64, wuv, wa = f64(kv), f64(w_uv), f64(w_a)
+    for seg in (0, 5, 7):                      # document 5 is the one cut by the two row ranges
+        lo = int(lay.seg_off[seg])
+        canon = np.array([0, 1, 127, 128, 129, 255, 256, 257, 1233, 1234, 1235, 2047, 4094, 4095])
+        want = oracle.mla_off_artifact(seg, f64(q_l_doc[torch.as_tensor(lo + canon, device="cuda")]), kv64, lay.seg_off,
+                                       lay.seg_delta, prof.local_heads, wuv, wa, prof.sm_scale, prof.rope_base,
+                                       prof.d_latent, rows=canon)
+        assert_close(f64(z_off[torch.as_tensor(lo + canon, device="cuda")]), want, f"z_off rows of document {seg}")

@@ -347,3 +347,66 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable(rk):
     O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
     ctx.rk_poll_status()
     assert_close(f64(O_g), exp["O_g"], "O_g after a timed-out launch")
+
+
+# -- offline side: MLA-Off artifact build (Algorithm 1) ----------------------------------------------------
+
+def _honest_artifact_oracle(w):
+    p, lay = w.profile, w.layout
+    z = np.zeros((lay.n_doc_rows, p.n_groups * p.o_rank))
+    q_all = f64(w.q_all)
+    for i in range(lay.n_segs):
+        if lay.seg_has_artifact[i]:
+            lo, hi = int(lay.seg_off[i]), int(lay.seg_off[i + 1])
+            z[lo:hi] = oracle.mla_off_artifact(i, q_all[lo:hi][:, p.local_heads], f64(w.kv), lay.seg_off, lay.seg_delta,
+                                               p.local_heads, f64(w.w_uv), f64(w.w_a), p.sm_scale, p.rope_base, p.d_latent)
+    return z
+
+
+@pytest.mark.parametrize("name", ["tiny", "ragged"])
+def test_mla_off_build_matches_checker(rk, name):
+    w = synth.make_workload("tiny", regime="sharp", with_q_all=True) if name == "tiny" else \
+        synth.make_custom([300, 77, 513], 50, n_heads=16, n_groups=2, o_rank=256, d_model=512, pct_bp=700, seed=15,
+                          with_q_all=True)
+    p, lay = w.profile, w.layout
+    want = _honest_artifact_oracle(w)
+    ctx, req = make(rk, w)
+    to_device(w)
+    n = lay.n_doc_rows
+    q_l_doc = w.q_all[:n][:, torch.as_tensor(p.local_heads.astype(np.int64), device="cuda")].contiguous()
+    z_off = ctx.rk_mla_off_build(req, w.kv, 0, n, q_l_doc, w.w_uv, w.w_a)
+    ctx.rk_poll_status()
+    assert_close(f64(z_off), want, "z_off")
+    # built in two row ranges that cut a document in the middle: same rows, same values
+    cut = n // 2 + 3
+    za = ctx.rk_mla_off_build(req, w.kv, 0, cut, q_l_doc[:cut].contiguous(), w.w_uv, w.w_a)
+    zb = ctx.rk_mla_off_build(req, w.kv, cut, n, q_l_doc[cut:].contiguous(), w.w_uv, w.w_a)
+    ctx.rk_poll_status()
+    assert_close(f64(torch.cat([za, zb])), want, "z_off in two ranges")
+
+
+def test_offline_then_online_chain_reuses_first_document_exactly(rk):
+    """GPU-built artifact -> GPU online layer.  Against the checker's expected MLA-Online output, and:
+    the document placed first in the request (delta = 0) was built in the very context it is used in,
+    so its rows equal full recomputation (all heads on all rows) even where they are not protected."""
+    w = synth.make_workload("tiny", regime="sharp", with_q_all=True)
+    p, lay = w.profile, w.layout
+    want_off = _honest_artifact_oracle(w)
+    exp = oracle_online(w, np.arange(lay.n_rows), z_off=want_off)
+    _, y_full = oracle.full_recompute_rows(np.arange(lay.n_rows), f64(w.q_all), f64(w.kv), lay.seg_off, lay.seg_delta,
+                                           f64(w.w_uv), f64(w.w_a), f64(w.w_b), p.sm_scale, p.rope_base, p.d_latent)
+    ctx, req = make(rk, w)
+    to_device(w)
+    n = lay.n_doc_rows
+    q_l_doc = w.q_all[:n][:, torch.as_tensor(p.local_heads.astype(np.int64), device="cuda")].contiguous()
+    z_off = ctx.rk_mla_off_build(req, w.kv, 0, n, q_l_doc, w.w_uv, w.w_a)
+    O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
+    z_on_g, z_on_l = ctx.rk_group_sliced_proj(req, O_g, O_l, w.w_uv, w.w_a)
+    z, y = ctx.rk_combine_offline(req, z_on_g, z_on_l, z_off, w.w_b)
+    ctx.rk_poll_status()
+    assert_close(f64(y), exp["y"], "y with the GPU-built artifact")
+    first = int(np.argmin(lay.seg_delta[:-1]))
+    lo, hi = int(lay.seg_off[first]), int(lay.seg_off[first + 1])
+    assert_close(f64(y[lo:hi]), y_full[lo:hi], "first document rows vs full recomputation")
+    inv = oracle.inverse_row_map(w.prot_rows, lay.n_rows)
+    assert_close(f64(y)[inv >= 0], y_full[inv >= 0], "protected rows vs full recomputation")
