@@ -220,9 +220,13 @@ typedef struct rk_layer_buffers {
   size_t workspace_bytes;
 } rk_layer_buffers;
 
-/* One whole layer from HOST inputs: copies kv, q_g, q_l, z_off host->device (pinned host
- * memory recommended), runs (2), (4), (5) on `stream`, copies y device->host and synchronises
- * the stream.  Weights stay resident on the device. */
+/* One whole layer from HOST inputs: copies kv, q_g, q_l, z_off host->device (use pinned host
+ * memory; pageable memory works but serialises), runs (2), (4), (5), copies y device->host and
+ * synchronises `stream`.  Weights stay resident on the device.  Copies that the running kernel
+ * does not need yet travel on an internal second stream beside it (the Local pass needs only kv
+ * and q_l; q_g and the artifact arrive meanwhile; y returns in row chunks behind the shared
+ * projection) and are ordered by device events, not by host polling (Section "Turning omitted
+ * work into latency reduction": prefetch stream guarded by device events). */
 rk_status rk_layer_host(rk_ctx* ctx, const rk_request* req, const void* kv_host, const void* q_g_host,
                         const void* q_l_host, const void* z_off_host, const void* W_uv, const void* W_a,
                         const void* W_b, const rk_layer_buffers* dev, void* y_host, void* stream);

@@ -33,6 +33,8 @@ struct rk_ctx {
   int off_uv_g = 0, off_uv_l = 0, off_wa_g = 0, off_wa_l = 0, off_wb = 0;
   unsigned long long wait_ns = 2000ull * 1000 * 1000;
   int attn_debug = 0;  // development switches of the attention kernel (rk_set_debug_flags)
+  cudaStream_t copy_stream = nullptr;  // rk_layer_host: copies that overlap the kernels
+  cudaEvent_t ev[8] = {nullptr};       // device-side ordering between the two streams (no host polling)
   PFN_encodeTiled encode = nullptr;
   mutable std::string err;
 };
@@ -212,6 +214,13 @@ rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
     return RK_ERR_CUDA;
   }
   ctx->n_pairs = attention_max_pairs(ctx->sm_count);
+  e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+  for (int i = 0; i < 8 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    rk_destroy(ctx);
+    return RK_ERR_CUDA;
+  }
 
   // GEMM batch tables (depend only on the head partition)
   const int G = prof->n_groups, L = (int)ctx->local_heads.size(), ro = prof->o_rank;
@@ -247,6 +256,9 @@ rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
 
 rk_status rk_destroy(rk_ctx* ctx) {
   if (!ctx) return RK_ERR_NULL;
+  for (int i = 0; i < 8; ++i)
+    if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   cudaFree(ctx->d_status);
   cudaFree(ctx->d_batches);
   delete ctx;
@@ -665,23 +677,63 @@ rk_status rk_layer_host(rk_ctx* ctx, const rk_request* rq, const void* kv_host, 
   if (rq->A > 0 && !q_l_host) return fail(ctx, RK_ERR_NULL, "q_l_host is required");
   if (rq->A < rq->T && !z_off_host) return fail(ctx, RK_ERR_NULL, "z_off_host is required");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  cudaStream_t cp = ctx->copy_stream;
   const int G = ctx->prof.n_groups, L = ctx->prof.n_heads - G;
+  const int64_t T = rq->T, dm = ctx->prof.d_model;
   const size_t width = (size_t)G * ctx->prof.o_rank;
-  cudaError_t e = cudaMemcpyAsync(dev->kv, kv_host, (size_t)rq->T * kDQK * 2, cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dev->q_g, q_g_host, (size_t)rq->T * G * kDQK * 2, cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess && rq->A > 0)
+  const bool has_l = rq->A > 0;
+  // The copy stream starts after everything already queued on `stream` (the staging buffers may
+  // still be in use by an earlier call) and runs beside the kernels from then on: the Local pass
+  // needs only kv and q_l, so q_g and the artifact travel while it computes; y goes back in row
+  // chunks while the shared projection of the next chunk runs.  Ordering is by device events.
+  cudaError_t e = cudaEventRecord(ctx->ev[0], st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(cp, ctx->ev[0], 0);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dev->kv, kv_host, (size_t)T * kDQK * 2, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && has_l)
     e = cudaMemcpyAsync(dev->q_l, q_l_host, (size_t)rq->A * L * kDQK * 2, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dev->q_g, q_g_host, (size_t)T * G * kDQK * 2, cudaMemcpyHostToDevice, cp);
+  if (e == cudaSuccess) e = cudaEventRecord(ctx->ev[1], cp);
   if (e == cudaSuccess && rq->n_off_rows > 0 && z_off_host)
-    e = cudaMemcpyAsync(dev->z_off, z_off_host, (size_t)rq->n_off_rows * width * 2, cudaMemcpyHostToDevice, st);
+    e = cudaMemcpyAsync(dev->z_off, z_off_host, (size_t)rq->n_off_rows * width * 2, cudaMemcpyHostToDevice, cp);
+  if (e == cudaSuccess) e = cudaEventRecord(ctx->ev[2], cp);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "host to device copy");
-  rk_status s = rk_mla_online_attn(ctx, rq, dev->kv, dev->q_g, rq->A > 0 ? dev->q_l : nullptr, dev->O_g, dev->lse_g,
-                                   rq->A > 0 ? dev->O_l : nullptr, rq->A > 0 ? dev->lse_l : nullptr, stream);
-  if (s == RK_OK)
-    s = rk_group_sliced_proj(ctx, rq, dev->O_g, rq->A > 0 ? dev->O_l : nullptr, W_uv, W_a, dev->z_on_g,
-                             rq->A > 0 ? dev->z_on_l : nullptr, dev->workspace, dev->workspace_bytes, stream);
-  if (s == RK_OK) s = rk_combine_offline(ctx, rq, dev->z_on_g, dev->z_on_l, dev->z_off, W_b, dev->z, dev->y, stream);
+  rk_status s = RK_OK;
+  if (has_l) s = rk_mla_online_attn(ctx, rq, dev->kv, nullptr, dev->q_l, nullptr, nullptr, dev->O_l, dev->lse_l, stream);
   if (s != RK_OK) return s;
-  e = cudaMemcpyAsync(y_host, dev->y, (size_t)rq->T * ctx->prof.d_model * 2, cudaMemcpyDeviceToHost, st);
+  e = cudaStreamWaitEvent(st, ctx->ev[1], 0);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
+  s = rk_mla_online_attn(ctx, rq, dev->kv, dev->q_g, nullptr, dev->O_g, dev->lse_g, nullptr, nullptr, stream);
+  if (s == RK_OK)
+    s = rk_group_sliced_proj(ctx, rq, dev->O_g, has_l ? dev->O_l : nullptr, W_uv, W_a, dev->z_on_g,
+                             has_l ? dev->z_on_l : nullptr, dev->workspace, dev->workspace_bytes, stream);
+  if (s != RK_OK) return s;
+  e = cudaStreamWaitEvent(st, ctx->ev[2], 0);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
+  // restore-and-replace + W_b in up to four row chunks; each chunk's y is copied out behind it
+  const int n_chunks = T >= 4 * 1024 ? 4 : 1;
+  const int64_t rows_per = ((T + n_chunks - 1) / n_chunks + 127) / 128 * 128;
+  const uint8_t* zg = reinterpret_cast<const uint8_t*>(dev->z_on_g);
+  const uint8_t* zo = reinterpret_cast<const uint8_t*>(dev->z_off);
+  uint8_t* zz = reinterpret_cast<uint8_t*>(dev->z);
+  uint8_t* yy = reinterpret_cast<uint8_t*>(dev->y);
+  for (int c = 0; c < n_chunks; ++c) {
+    const int64_t r0 = c * rows_per, r1 = std::min<int64_t>(T, r0 + rows_per);
+    if (r0 >= r1) break;
+    e = launch_combine(zg + r0 * width * 2, dev->z_on_l, zo ? zo + r0 * width * 2 : nullptr, rq->d_inv_map + r0, r1 - r0,
+                       (int64_t)width, zz + r0 * width * 2, ctx->sm_count, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "combine launch");
+    s = run_gemm(ctx, zz + r0 * width * 2, r1 - r0, (int64_t)width, W_b, dm, (int64_t)width, yy + r0 * dm * 2, dm,
+                 (int)(r1 - r0), (int)dm, (int)width, ctx->off_wb, 1, st);
+    if (s != RK_OK) return s;
+    e = cudaEventRecord(ctx->ev[3 + c], st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(cp, ctx->ev[3 + c], 0);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(reinterpret_cast<uint8_t*>(y_host) + r0 * dm * 2, yy + r0 * dm * 2, (size_t)(r1 - r0) * dm * 2,
+                          cudaMemcpyDeviceToHost, cp);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "device to host copy");
+  }
+  e = cudaEventRecord(ctx->ev[7], cp);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(st, ctx->ev[7], 0);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "device to host copy");
 }
