@@ -31,6 +31,14 @@ from paper_2609_07008_b200 import synth  # noqa: E402
 from paper_2609_07008_b200 import dist as rkdist  # noqa: E402
 
 FLOP_PER_PAIR = 2 * 576 + 2 * 512     # QK^T over 576 + PV over 512 per visible (row, key, head)
+# dram__bytes_read.sum + dram__bytes_write.sum of the attention kernel's two launches per step, from the
+# one-pass ncu captures summarised under profiles/ (bytes per step; None where no capture exists)
+PROFILED_DRAM_TRAFFIC = {
+    "flash256k": dict(bytes=37.80e9 + 9.22e9, algorithmic=4.91e9 + 1.20e9,
+                      source="profiles/attn_kernel_flash256k_dram_traffic.md"),
+    "flash1": dict(bytes=(355.0e6 + 234.6e6) + (180.5e6 + 84.0e6), algorithmic=(350.3e6 + 277.9e6) + (168.4e6 + 115.5e6),
+                   source="profiles/attn_kernel_flash1_ncu_full.md"),
+}
 L2_BYTES = 126 * 1024 * 1024
 
 
@@ -363,6 +371,29 @@ def main():
     if not args.no_aux and rank == 0:
         aux = time_stream_kernels(ctx, req, w, prof, lay, dev)
 
+    # where the rest of the step goes (instrumentation pass, not the timed region)
+    breakdown = None
+    if rank == 0:
+        def ev_ms(fn, reps=3):
+            fn()
+            out = []
+            for _ in range(reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); fn(); b.record(stream); torch.cuda.synchronize()
+                out.append(a.elapsed_time(b))
+            return float(np.mean(out))
+        t_proj = ev_ms(lambda: ctx.rk_group_sliced_proj(req, bufs["O_g"], bufs["O_l"], w.w_uv, w.w_a, bufs["z_on_g"],
+                                                        bufs["z_on_l"], bufs["workspace"]))
+        t_comb = ev_ms(lambda: ctx.rk_combine_offline(req, bufs["z_on_g"], bufs["z_on_l"], w.z_off, None, bufs["z"]))
+        t_cwb = ev_ms(lambda: ctx.rk_combine_offline(req, bufs["z_on_g"], bufs["z_on_l"], w.z_off, w.w_b, bufs["z"],
+                                                     bufs["y"]))
+        width = prof.n_groups * prof.o_rank
+        comb_bytes = 3 * req.T * width * 2
+        breakdown = dict(sliced_proj_ms=t_proj, sliced_proj_tflops=fl_proj / t_proj / 1e9,
+                         combine_ms=t_comb, combine_gbs=comb_bytes / t_comb / 1e6,
+                         wb_gemm_ms=t_cwb - t_comb, wb_gemm_tflops=fl_wb / (t_cwb - t_comb) / 1e9)
+        ctx.rk_poll_status()
+
     offline = None
     if args.with_offline and rank == 0:
         offline = time_offline_build(ctx, req, w, prof, lay, dev)
@@ -378,7 +409,10 @@ def main():
                     frac=attn_tflops / peaks["bf16_sustained"], peak_source=peaks["source"] + " sustained bf16",
                     frac_of_burst=attn_tflops / peaks["bf16_burst"], frac_of_nominal=attn_tflops / 2250.0,
                     launches_per_step=2, ms_per_step=float(np.mean(attn_ms)),
-                    ms_global_pass=float(np.mean(attn_g_ms)), traffic=None)
+                    ms_global_pass=float(np.mean(attn_g_ms)),
+                    traffic=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("bytes"),
+                    traffic_note=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("source", "no ncu capture of this workload"),
+                    algorithmic_dram_bytes=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("algorithmic"))
     rest_tflops = (fl_proj + fl_wb) / (np.mean(rest_ms) * 1e-3) / 1e12
 
     cpu_baseline = None
@@ -406,6 +440,8 @@ def main():
                             flops_attn=fl_attn, flops_proj=fl_proj + fl_wb),
                 clocks=clocks, e2e=e2e, gpu_launches=launches_per_step * args.steps, roofline=roofline,
                 proj_tflops=rest_tflops, proj_ms_per_step=float(np.mean(rest_ms)), cpu_baseline=cpu_baseline)
+    if breakdown:
+        line["projection_breakdown"] = breakdown
     if offline:
         line["offline_build"] = offline
     if aux:

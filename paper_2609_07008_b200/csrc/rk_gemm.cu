@@ -1,8 +1,9 @@
 // Batched dense projection  C[M, N] = A[M, K] * B[N, K]^T  (bf16 operands, fp32 accumulation in
 // TMEM, bf16 result) used for the per-head up-projection W_uv, the group-aligned slices of the
 // first output projection W_a (Eq. offonline) and the shared second projection W_b
-// (Eq. factorization).  One CTA per 128 x BN output tile; TMA -> 128B-swizzled shared memory
-// -> tcgen05.mma (cta_group::1, M=128, N=BN, K=16) -> tcgen05.ld epilogue.
+// (Eq. factorization).  Persistent CTAs over 128 x BN output tiles; TMA -> 128B-swizzled shared
+// memory -> tcgen05.mma (cta_group::1, M=128, N=BN, K=16) into one of two TMEM accumulators ->
+// tcgen05.ld epilogue that overlaps the next tile's main loop.
 //
 // A batch (blockIdx.z) selects column/row blocks of the 2-D operands: a head's or a group's
 // block.  `b_skip` opens a 128-column hole in B's K axis so that the seven Local slices of a
@@ -17,6 +18,7 @@ namespace {
 constexpr int kStages = 4;
 constexpr int kBM = 128;
 constexpr int kBK = 64;
+constexpr int kGemmThreads = 256;
 
 template <int BN>
 struct GemmSmem {
@@ -24,15 +26,19 @@ struct GemmSmem {
   static constexpr uint32_t kBBytes = BN * kBK * 2;
   static constexpr uint32_t kStageBytes = kABytes + kBBytes;
   static constexpr uint32_t kOffBars = kStages * kStageBytes;
-  static constexpr uint32_t kOffTmemPtr = kOffBars + (2 * kStages + 1) * 8;
+  // full[kStages], empty[kStages], acc_full[2], acc_empty[2]
+  static constexpr uint32_t kOffTmemPtr = kOffBars + (2 * kStages + 4) * 8;
   static constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
   static constexpr uint32_t kBytes = kOffAbort + 8 + 1024;
 };
 
-enum { WG_FULL = 31, WG_EMPTY, WG_ACC };
+enum { WG_FULL = 31, WG_EMPTY, WG_ACC_FULL, WG_ACC_EMPTY };
 
+// Persistent: each CTA walks output tiles t = blockIdx.x, + gridDim.x, ... (column tile fastest, so
+// CTAs running at the same time share A row blocks and the whole of B through L2).  Two TMEM
+// accumulator buffers let the epilogue of tile i overlap the main loop of tile i + 1.
 template <int BN>
-__global__ void __launch_bounds__(256, 1) rk_gemm_kernel(const __grid_constant__ GemmParams p) {
+__global__ void __launch_bounds__(kGemmThreads, 1) rk_gemm_kernel(const __grid_constant__ GemmParams p) {
   using S = GemmSmem<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -41,15 +47,18 @@ __global__ void __launch_bounds__(256, 1) rk_gemm_kernel(const __grid_constant__
   const int lane = threadIdx.x & 31;
   auto full_bar = [&](int s) -> uint32_t { return smem_base + S::kOffBars + 8u * s; };
   auto empty_bar = [&](int s) -> uint32_t { return smem_base + S::kOffBars + 8u * (kStages + s); };
-  const uint32_t acc_bar = smem_base + S::kOffBars + 8u * (2 * kStages);
+  auto acc_full_bar = [&](int b) -> uint32_t { return smem_base + S::kOffBars + 8u * (2 * kStages + b); };
+  auto acc_empty_bar = [&](int b) -> uint32_t { return smem_base + S::kOffBars + 8u * (2 * kStages + 2 + b); };
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::kOffAbort);
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + S::kOffTmemPtr);
   const uint64_t limit = p.wait_ns;
 
-  const int n0 = blockIdx.x * BN;
-  const int m0 = blockIdx.y * kBM;
-  const GemmBatch bt = p.batches[blockIdx.z];
+  const int n_tiles_n = (p.N + BN - 1) / BN;
+  const int n_tiles_m = (p.M + kBM - 1) / kBM;
+  const int tiles_per_batch = n_tiles_n * n_tiles_m;
+  const int n_tiles = tiles_per_batch * p.n_batches;
   const int k_chunks = p.K / kBK;
+  constexpr uint32_t kTmemCols = 2 * BN;  // 256 or 512: power of two
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -57,12 +66,15 @@ __global__ void __launch_bounds__(256, 1) rk_gemm_kernel(const __grid_constant__
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
-    mbar_init(acc_bar, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(acc_full_bar(b), 1);
+      mbar_init(acc_empty_bar(b), 4);  // one arrival per epilogue warp
+    }
     fence_mbar_init_cluster();
   }
   if (warp == 0) {
     __syncwarp();
-    tmem_alloc<1>(smem_base + S::kOffTmemPtr, BN);
+    tmem_alloc<1>(smem_base + S::kOffTmemPtr, kTmemCols);
     tmem_relinquish<1>();
   }
   tc_fence_before_sync();
@@ -71,55 +83,94 @@ __global__ void __launch_bounds__(256, 1) rk_gemm_kernel(const __grid_constant__
   const uint32_t tmem_base = *tmem_ptr_smem;
 
   if (warp == 0) {
+    // ---- TMA producer (whole warp loops, one elected lane issues) ----
     if (lane == 0) {
       tma_prefetch_desc(&p.tm_a);
       tma_prefetch_desc(&p.tm_b);
-      bool ok = true;
-      for (int kc = 0; kc < k_chunks && ok; ++kc) {
-        const int s = kc % kStages;
-        const uint32_t use = kc / kStages;
-        if (use > 0)
-          ok = mbar_wait_bounded<false>(empty_bar(s), (use - 1) & 1u, limit, abort_flag, p.status, WG_EMPTY, kc);
+    }
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+      const int batch = t / tiles_per_batch;
+      const int rem = t - batch * tiles_per_batch;
+      const int m0 = (rem / n_tiles_n) * kBM, n0 = (rem % n_tiles_n) * BN;
+      const GemmBatch bt = p.batches[batch];
+      for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
+        const uint32_t s = it % kStages;
+        if (it >= (uint32_t)kStages)
+          ok = mbar_wait_bounded<false>(empty_bar(s), ((it / kStages) & 1u) ^ 1u, limit, abort_flag, p.status, WG_EMPTY, t);
         if (!ok) break;
-        mbar_arrive_expect_tx(full_bar(s), S::kStageBytes);
-        const int k = kc * kBK;
-        const int bk = bt.b_col0 + k + (k >= bt.b_skip ? 128 : 0);
-        const uint32_t a_dst = smem_base + s * S::kStageBytes;
-        tma_load_2d(a_dst, &p.tm_a, full_bar(s), bt.a_col0 + k, m0);
-        tma_load_2d(a_dst + S::kABytes, &p.tm_b, full_bar(s), bk, bt.b_row0 + n0);
+        if (elect_one()) {
+          mbar_arrive_expect_tx(full_bar(s), S::kStageBytes);
+          const int k = kc * kBK;
+          const int bk = bt.b_col0 + k + (k >= bt.b_skip ? 128 : 0);
+          const uint32_t a_dst = smem_base + s * S::kStageBytes;
+          tma_load_2d(a_dst, &p.tm_a, full_bar(s), bt.a_col0 + k, m0);
+          tma_load_2d(a_dst + S::kABytes, &p.tm_b, full_bar(s), bk, bt.b_row0 + n0);
+        }
+        __syncwarp();
+      }
+    }
+    // drain: the tensor core must have released every stage this CTA filled
+    for (uint32_t back = 1; back <= (uint32_t)kStages && ok; ++back) {
+      if (it >= back) {
+        const uint32_t u = it - back;
+        ok = mbar_wait_bounded<false>(empty_bar(u % kStages), (u / kStages) & 1u, limit, abort_flag, p.status, WG_EMPTY, -1);
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN, 0, 0);
-      bool ok = true;
-      for (int kc = 0; kc < k_chunks && ok; ++kc) {
-        const int s = kc % kStages;
-        ok = mbar_wait_bounded<false>(full_bar(s), (kc / kStages) & 1u, limit, abort_flag, p.status, WG_FULL, kc);
+    // ---- UMMA issuer (whole warp loops, one elected lane issues 4 MMAs + commit per stage) ----
+    constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN, 0, 0);
+    uint32_t it = 0, tile_i = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
+      const uint32_t b = tile_i & 1u;
+      if (tile_i >= 2) {
+        ok = mbar_wait_bounded<false>(acc_empty_bar(b), ((tile_i >> 1) & 1u) ^ 1u, limit, abort_flag, p.status,
+                                      WG_ACC_EMPTY, t);
         if (!ok) break;
         tc_fence_after_sync();
+      }
+      const uint32_t tmem_acc = tmem_base + b * BN;
+      for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
+        const uint32_t s = it % kStages;
+        ok = mbar_wait_bounded<false>(full_bar(s), (it / kStages) & 1u, limit, abort_flag, p.status, WG_FULL, t);
+        if (!ok) break;
         const uint32_t a_addr = smem_base + s * S::kStageBytes;
         const uint32_t b_addr = a_addr + S::kABytes;
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_f16<1>(tmem_base, umma_desc_sw128(a_addr + k * 32, 16, 1024), umma_desc_sw128(b_addr + k * 32, 16, 1024),
-                      idesc, (kc > 0 || k > 0) ? 1u : 0u);
-        umma_commit_1(empty_bar(s));
+          for (int k = 0; k < 4; ++k)
+            umma_f16<1>(tmem_acc, umma_desc_sw128(a_addr + k * 32, 16, 1024), umma_desc_sw128(b_addr + k * 32, 16, 1024),
+                        idesc, (kc > 0 || k > 0) ? 1u : 0u);
+          umma_commit_1(empty_bar(s));
+          if (kc == k_chunks - 1) umma_commit_1(acc_full_bar(b));
+        }
+        __syncwarp();
       }
-      if (ok) umma_commit_1(acc_bar);
     }
   } else if (warp >= 4) {
+    // ---- epilogue: TMEM -> registers -> bf16 -> global, one row per thread ----
     const int L = threadIdx.x - 128;
     const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
-    bool ok = mbar_wait_bounded<false>(acc_bar, 0, limit, abort_flag, p.status, WG_ACC, 0);
-    if (ok) {
+    uint32_t tile_i = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
+      const uint32_t b = tile_i & 1u;
+      const int batch = t / tiles_per_batch;
+      const int rem = t - batch * tiles_per_batch;
+      const int m0 = (rem / n_tiles_n) * kBM, n0 = (rem % n_tiles_n) * BN;
+      const GemmBatch bt = p.batches[batch];
+      ok = mbar_wait_bounded<false>(acc_full_bar(b), (tile_i >> 1) & 1u, limit, abort_flag, p.status, WG_ACC_FULL, t);
+      if (!ok) break;
       tc_fence_after_sync();
       const int row = m0 + L;
-      __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(p.C) + (size_t)(row < p.M ? row : 0) * p.ldc + bt.c_col0 + n0;
+      __nv_bfloat16* crow =
+          reinterpret_cast<__nv_bfloat16*>(p.C) + (size_t)(row < p.M ? row : 0) * p.ldc + bt.c_col0 + n0;
 #pragma unroll 1
       for (int cc = 0; cc < BN; cc += 32) {
         uint32_t o[32];
-        tmem_ld_x32(tmem_base + lane_base + cc, o);
+        tmem_ld_x32(tmem_base + lane_base + b * BN + cc, o);
         tmem_wait_ld();
         if (row < p.M && n0 + cc < p.N) {
           uint4* dst = reinterpret_cast<uint4*>(crow + cc);
@@ -134,6 +185,9 @@ __global__ void __launch_bounds__(256, 1) rk_gemm_kernel(const __grid_constant__
           }
         }
       }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty_bar(b));
     }
   }
   __syncwarp();
@@ -141,7 +195,7 @@ __global__ void __launch_bounds__(256, 1) rk_gemm_kernel(const __grid_constant__
   __syncthreads();
   if (warp == 0) {
     __syncwarp();
-    tmem_dealloc<1>(tmem_base, BN);
+    tmem_dealloc<1>(tmem_base, kTmemCols);
   }
 }
 
@@ -155,12 +209,14 @@ cudaError_t gemm_setup() {
                               (int)GemmSmem<256>::kBytes);
 }
 
-cudaError_t launch_gemm(const GemmParams& p, int bn, cudaStream_t stream) {
-  dim3 grid((p.N + bn - 1) / bn, (p.M + kBM - 1) / kBM, p.n_batches);
+cudaError_t launch_gemm(const GemmParams& p, int bn, int sm_count, cudaStream_t stream) {
+  const long long tiles = (long long)((p.N + bn - 1) / bn) * ((p.M + kBM - 1) / kBM) * p.n_batches;
+  if (tiles <= 0) return cudaSuccess;
+  const int grid = (int)(tiles < sm_count ? tiles : sm_count);
   if (bn == 128)
-    rk_gemm_kernel<128><<<grid, 256, GemmSmem<128>::kBytes, stream>>>(p);
+    rk_gemm_kernel<128><<<grid, kGemmThreads, GemmSmem<128>::kBytes, stream>>>(p);
   else
-    rk_gemm_kernel<256><<<grid, 256, GemmSmem<256>::kBytes, stream>>>(p);
+    rk_gemm_kernel<256><<<grid, kGemmThreads, GemmSmem<256>::kBytes, stream>>>(p);
   return cudaGetLastError();
 }
 

@@ -608,7 +608,7 @@ static rk_status run_gemm(rk_ctx* ctx, const void* A, int64_t a_rows, int64_t a_
   p.N = N;
   p.K = K;
   p.n_batches = n_batches;
-  cudaError_t e = launch_gemm(p, bn, st);
+  cudaError_t e = launch_gemm(p, bn, ctx->sm_count, st);
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "gemm launch");
 }
 

@@ -74,7 +74,7 @@ struct GemmParams {
   int32_t n_batches;
 };
 
-cudaError_t launch_gemm(const GemmParams& p, int bn, cudaStream_t stream);
+cudaError_t launch_gemm(const GemmParams& p, int bn, int sm_count, cudaStream_t stream);
 cudaError_t gemm_setup();
 
 // ---- streaming kernels -----------------------------------------------------------------------
