@@ -334,20 +334,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             if (elect_one()) {
               if (st < 4) {
                 const uint32_t a_addr = q_base + 2 * st * kQChunkBytes;
+                // descriptors differ only in the start-address field (16-byte units): add constants
+                const uint64_t da = umma_desc_sw128(a_addr, 16, 1024), db = umma_desc_sw128(b_addr, 16, 1024);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                  umma_f16<2>(tmem_s, umma_desc_sw128(a_addr + (k >> 2) * kQChunkBytes + (k & 3) * 32, 16, 1024),
-                              umma_desc_sw128(b_addr + (k >> 2) * kChunkBytes + (k & 3) * 32, 16, 1024), kIdescQK,
+                  umma_f16<2>(tmem_s, da + (uint64_t)(((k >> 2) * kQChunkBytes + (k & 3) * 32) >> 4),
+                              db + (uint64_t)(((k >> 2) * kChunkBytes + (k & 3) * 32) >> 4), kIdescQK,
                               (st > 0 || k > 0) ? 1u : 0u);
                 }
                 umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
               } else {
                 const uint32_t a_addr = smem_base + kOffQRot + rb * kQChunkBytes;
+                const uint64_t da = umma_desc_sw128(a_addr, 16, 1024), db = umma_desc_sw128(b_addr, 16, 1024);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  umma_f16<2>(tmem_s, umma_desc_sw128(a_addr + k * 32, 16, 1024),
-                              umma_desc_sw128(b_addr + k * 32, 16, 1024), kIdescQK, 1u);
-                }
+                for (int k = 0; k < 4; ++k) umma_f16<2>(tmem_s, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), kIdescQK, 1u);
                 umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
                 umma_commit_2_mc(bar(kBarSFull + (kt_issued & 1)), 3);
                 if (last_of_seg) umma_commit_2_mc(bar(kBarQrFree + rb), 3);
@@ -375,12 +375,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             const uint32_t b_addr = smem_base + kOffRing + s * kStageBytes;
             const uint32_t tmem_o = tmem_base + kColO + (uint32_t)h * 128u;
             if (elect_one()) {
+              const uint64_t da = umma_desc_sw128(p_base + 2 * kh * kQChunkBytes, 16, 1024);
+              const uint64_t db = umma_desc_sw128(b_addr, kChunkBytes, 1024);
 #pragma unroll
               for (int k = 0; k < 8; ++k) {
-                const uint32_t a_addr = p_base + (2 * kh + (k >> 2)) * kQChunkBytes + (k & 3) * 32;
-                umma_f16<2>(tmem_o, umma_desc_sw128(a_addr, 16, 1024),
-                            umma_desc_sw128(b_addr + k * 2048, kChunkBytes, 1024), kIdescPV,
-                            (kt_pv > 0 || kh > 0 || k > 0) ? 1u : 0u);
+                umma_f16<2>(tmem_o, da + (uint64_t)(((k >> 2) * kQChunkBytes + (k & 3) * 32) >> 4),
+                            db + (uint64_t)((k * 2048) >> 4), kIdescPV, (kt_pv > 0 || kh > 0 || k > 0) ? 1u : 0u);
               }
               umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
               if (q == 3) umma_commit_2_mc(bar(kBarPvDone), 3);
