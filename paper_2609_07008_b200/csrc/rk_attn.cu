@@ -304,7 +304,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     // ------------------------------ UMMA issuer (leader CTA; whole warp loops, elected lane issues) --
     if (leader) {
       RingPos rp;
-      uint32_t qr_ready_phase[2] = {0, 0};
+      uint32_t qr_ready_phases = 0;  // bit rb = parity to wait for
       uint32_t p_ready_phase = 0;
       uint32_t qr_use = 0;  // counts rope-buffer uses across tiles
       bool ok = true;
@@ -319,10 +319,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
 
         auto issue_qk = [&](bool first_of_seg, bool last_of_seg, uint32_t rb) -> bool {
           if (first_of_seg) {
-            if (!mbar_wait_bounded<true>(bar(kBarQrReady + rb), qr_ready_phase[rb], limit, abort_flag, p.status,
-                                         W_QRREADY, w))
+            if (!mbar_wait_bounded<true>(bar(kBarQrReady + rb), (qr_ready_phases >> rb) & 1u, limit, abort_flag,
+                                         p.status, W_QRREADY, w))
               return false;
-            qr_ready_phase[rb] ^= 1;
+            qr_ready_phases ^= (1u << rb);
           }
           const uint32_t tmem_s = tmem_base + kColS + (uint32_t)(kt_issued & 1) * 128u;
 #pragma unroll 1
@@ -409,7 +409,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
   } else if (warp == 2) {
     // ------------------------------ query relocation ----------------------------------------
     uint32_t qfull_phase = 0;
-    uint32_t qr_free_phase[2] = {0, 0};
+    uint32_t qr_free_phases = 0;  // bit rb = parity to wait for
     uint32_t qr_use = 0;
     bool ok = true;
     for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
@@ -420,9 +420,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       while (ok && it.next()) {
         const uint32_t rb = qr_use & 1u;
         if (qr_use >= 2) {
-          ok = mbar_wait_bounded<true>(bar(kBarQrFree + rb), qr_free_phase[rb], limit, abort_flag, p.status,
+          ok = mbar_wait_bounded<true>(bar(kBarQrFree + rb), (qr_free_phases >> rb) & 1u, limit, abort_flag, p.status,
                                        W_QRFREE, w);
-          qr_free_phase[rb] ^= 1;
+          qr_free_phases ^= (1u << rb);
           if (!ok) break;
         }
         ++qr_use;
@@ -456,9 +456,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     if (lane == 0) {
       for (uint32_t u = (qr_use >= 2 ? qr_use - 2 : 0); u < qr_use && ok; ++u) {
         const uint32_t rb = u & 1u;
-        ok = mbar_wait_bounded<true>(bar(kBarQrFree + rb), qr_free_phase[rb], limit, abort_flag, p.status, W_DRAIN,
-                                     100 + (int)rb);
-        qr_free_phase[rb] ^= 1;
+        ok = mbar_wait_bounded<true>(bar(kBarQrFree + rb), (qr_free_phases >> rb) & 1u, limit, abort_flag, p.status,
+                                     W_DRAIN, 100 + (int)rb);
+        qr_free_phases ^= (1u << rb);
       }
     }
   } else if (warp >= 4) {
@@ -475,7 +475,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     const uint32_t lane_base = ((uint32_t)((sw & 3) * 32)) << 16;
     volatile unsigned long long* xbuf = reinterpret_cast<volatile unsigned long long*>(smem + kOffXchg);
     uint32_t xseq = 0;  // exchange sequence number
-    uint32_t s_full_phase[2] = {0, 0};
+    uint32_t s_full_phases = 0;  // bit b = parity to wait for
     uint32_t pv_done_phase = 0;
     bool ok = true;
     const float scale = p.scale_log2;
@@ -508,8 +508,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           int nv = lim - (kb + part * 64) + 1;
           nv = nv < 0 ? 0 : (nv > 64 ? 64 : nv);
           const int b = kt & 1;
-          ok = mbar_wait_bounded<false>(bar(kBarSFull + b), s_full_phase[b], limit, abort_flag, p.status, W_SFULL, w);
-          s_full_phase[b] ^= 1;
+          ok = mbar_wait_bounded<false>(bar(kBarSFull + b), (s_full_phases >> b) & 1u, limit, abort_flag, p.status,
+                                        W_SFULL, w);
+          s_full_phases ^= (1u << b);
           if (!ok) break;
           tc_fence_after_sync();
           if (p.debug & 1) {
