@@ -158,7 +158,8 @@ def run_reference(args, rank, world):
     pg = int(np.searchsorted(srt, pos, side="right").sum())
     pl = int(np.searchsorted(srt, pos[prot], side="right").sum())
     all_pairs = prof.n_groups * pg + prof.n_local * pl
-    rows = pick_oracle_rows(w, args.oracle_pairs)
+    # every step is one bounded sample; a third of the cpu_baseline budget keeps W + K steps within minutes
+    rows = pick_oracle_rows(w, max(1, args.oracle_pairs // 3))
     times, pairs = [], 0
     for i in range(args.warmup + args.steps):
         dt, pairs, _ = oracle_sample_run(w, rows)
@@ -276,6 +277,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-aux", action="store_true", help="skip the standalone relocation / merge timings")
     ap.add_argument("--with-offline", action="store_true", help="also time the offline artifact build")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="independent layer invocations per step (own values and protected rows each; "
+                         "default 37 for flash32k, the 3F-37R-3F stack, else 1)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rk" else args.warmup
 
@@ -290,33 +294,48 @@ def main():
     from paper_2609_07008_b200 import binding as rk   # raises if librk.so is missing: no fallback
 
     name = args.config
-    prof, lay, prot = synth.make_geometry(name)
-    # every rank gets its own request values (independent requests, same shape)
-    w = synth.make_tensors(name, prof, lay, prot, rkdist.rank_seed(synth.CONFIGS[name]["seed"], rank), device=dev,
-                           regime=args.regime)
-    ctx = rk.Context.from_profile(prof)
-    if os.environ.get("RK_DEBUG_FLAGS"):      # timing experiments only; results are meaningless then
-        ctx.rk_set_debug_flags(int(os.environ["RK_DEBUG_FLAGS"]))
-    req = ctx.rk_request_create(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, prot)
-    bufs = ctx.alloc_layer_buffers(req, dev)
-    fl_attn, fl_proj, fl_wb = algorithmic_flops(prof, req)
-    in_bytes = sum(t.numel() * t.element_size() for t in (w.kv, w.q_g, w.q_l, w.z_off))
+    n_layers = args.layers or (synth.N_LAYERS_FLASH32K if name == "flash32k" else 1)
+    ctx = None
+    layers = []          # (workload, request) per layer: same layout, own values, own protected rows
+    for l in range(n_layers):
+        prof, lay, prot = synth.make_geometry(name, layer=l)
+        # every rank gets its own request values (independent requests, same shape)
+        wl = synth.make_tensors(name, prof, lay, prot, rkdist.rank_seed(synth.CONFIGS[name]["seed"], rank) + 7 * l,
+                                device=dev, regime=args.regime)
+        if ctx is None:
+            ctx = rk.Context.from_profile(prof)
+            if os.environ.get("RK_DEBUG_FLAGS"):      # timing experiments only; results are meaningless then
+                ctx.rk_set_debug_flags(int(os.environ["RK_DEBUG_FLAGS"]))
+        layers.append((wl, ctx.rk_request_create(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, prot)))
+    w, req = layers[0]
+    prof, lay = w.profile, w.layout
+    big = max(layers, key=lambda t: t[1].A)[1]
+    bufs = ctx.alloc_layer_buffers(big, dev)          # staging/outputs shared by the layers (they run in sequence)
+    fl_attn = fl_proj = fl_wb = 0
+    for _, r in layers:
+        a, b, c = algorithmic_flops(prof, r)
+        fl_attn, fl_proj, fl_wb = fl_attn + a, fl_proj + b, fl_wb + c
+    in_bytes = sum(t.numel() * t.element_size() for wl, _ in layers for t in (wl.kv, wl.q_g, wl.q_l, wl.z_off))
     need_flush = in_bytes < 4 * L2_BYTES
     flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if need_flush else None
     stream = torch.cuda.current_stream()
 
-    def step(ev=None):
+    def run_layer(wl, r, ev=None):
         if ev: ev[0].record(stream)
-        ctx.rk_mla_online_attn(req, w.kv, w.q_g, None, bufs["O_g"], bufs["lse_g"], None, None)
+        ctx.rk_mla_online_attn(r, wl.kv, wl.q_g, None, bufs["O_g"], bufs["lse_g"], None, None)
         if ev: ev[1].record(stream)
-        ctx.rk_mla_online_attn(req, w.kv, None, w.q_l, None, None, bufs["O_l"], bufs["lse_l"])
+        ctx.rk_mla_online_attn(r, wl.kv, None, wl.q_l, None, None, bufs["O_l"], bufs["lse_l"])
         if ev: ev[2].record(stream)
-        ctx.rk_group_sliced_proj(req, bufs["O_g"], bufs["O_l"], w.w_uv, w.w_a, bufs["z_on_g"], bufs["z_on_l"],
+        ctx.rk_group_sliced_proj(r, bufs["O_g"], bufs["O_l"], wl.w_uv, wl.w_a, bufs["z_on_g"], bufs["z_on_l"],
                                  bufs["workspace"])
-        ctx.rk_combine_offline(req, bufs["z_on_g"], bufs["z_on_l"], w.z_off, w.w_b, bufs["z"], bufs["y"])
+        ctx.rk_combine_offline(r, bufs["z_on_g"], bufs["z_on_l"], wl.z_off, wl.w_b, bufs["z"], bufs["y"])
         if ev: ev[3].record(stream)
 
-    launches_per_step = 2 + 4 + 1 + 1   # attention x2, projection GEMMs x4, combine, W_b GEMM
+    def step(ev=None):
+        for i, (wl, r) in enumerate(layers):
+            run_layer(wl, r, ev[i] if ev else None)
+
+    launches_per_step = (2 + 4 + 1 + 1) * n_layers   # per layer: attention x2, projection GEMMs x4, combine, W_b
 
     for _ in range(args.warmup):
         step()
@@ -326,7 +345,8 @@ def main():
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    evs = [[[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_layers)]
+           for _ in range(args.steps)]
     rkdist.barrier()
     torch.cuda.synchronize()
     for i in range(args.steps):
@@ -336,10 +356,10 @@ def main():
     rkdist.barrier()
     sampler.stop_flag = True
     ctx.rk_poll_status()
-    step_ms = [evs[i][0].elapsed_time(evs[i][3]) for i in range(args.steps)]
-    attn_ms = [evs[i][0].elapsed_time(evs[i][2]) for i in range(args.steps)]
-    attn_g_ms = [evs[i][0].elapsed_time(evs[i][1]) for i in range(args.steps)]
-    rest_ms = [evs[i][2].elapsed_time(evs[i][3]) for i in range(args.steps)]
+    step_ms = [evs[i][0][0].elapsed_time(evs[i][-1][3]) for i in range(args.steps)]
+    attn_ms = [sum(e[0].elapsed_time(e[2]) for e in evs[i]) for i in range(args.steps)]
+    attn_g_ms = [sum(e[0].elapsed_time(e[1]) for e in evs[i]) for i in range(args.steps)]
+    rest_ms = [sum(e[2].elapsed_time(e[3]) for e in evs[i]) for i in range(args.steps)]
     total_ms = float(sum(step_ms))
     total_ms_max = rkdist.max_over_ranks(total_ms, dev)
     sampler.join(timeout=2)
@@ -349,22 +369,27 @@ def main():
     e2e = None
     if not args.no_e2e:
         pin = lambda x: x.to("cpu").pin_memory()
-        hk, hqg, hql, hzo = pin(w.kv), pin(w.q_g), pin(w.q_l), pin(w.z_off)
+        host = [(pin(wl.kv), pin(wl.q_g), pin(wl.q_l), pin(wl.z_off)) for wl, _ in layers]
         y_h = torch.empty((req.T, prof.d_model), dtype=torch.bfloat16).pin_memory()
-        ctx.rk_layer_host(req, hk, hqg, hql, hzo, w.w_uv, w.w_a, w.w_b, bufs, y_h)   # warm-up
+
+        def e2e_step():
+            for (wl, r), (hk, hqg, hql, hzo) in zip(layers, host):
+                ctx.rk_layer_host(r, hk, hqg, hql, hzo, wl.w_uv, wl.w_a, wl.w_b, bufs, y_h)
+
+        e2e_step()   # warm-up
         rkdist.barrier()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         for _ in range(args.e2e_steps):
-            ctx.rk_layer_host(req, hk, hqg, hql, hzo, w.w_uv, w.w_a, w.w_b, bufs, y_h)
+            e2e_step()
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0)
         e2e_max = rkdist.max_over_ranks(e2e_s, dev)
         ctx.rk_poll_status()
-        e2e = dict(value=rkdist.aggregate_throughput(req.T, args.e2e_steps, world, e2e_max), unit="tokens/s",
-                   h2d_bytes_per_step=int(in_bytes), d2h_bytes_per_step=int(y_h.numel() * 2),
+        e2e = dict(value=rkdist.aggregate_throughput(req.T * n_layers, args.e2e_steps, world, e2e_max),
+                   unit="tokens/s", h2d_bytes_per_step=int(in_bytes), d2h_bytes_per_step=int(y_h.numel() * 2 * n_layers),
                    ms_per_step=e2e_max * 1e3 / args.e2e_steps)
-        del hk, hqg, hql, hzo
+        del host
 
     # standalone HBM-bound calls (not part of the step): relocation and merge against copy bandwidth
     aux = None
@@ -408,7 +433,7 @@ def main():
                     achieved=attn_tflops, peak=peaks["bf16_sustained"], unit="TFLOP/s",
                     frac=attn_tflops / peaks["bf16_sustained"], peak_source=peaks["source"] + " sustained bf16",
                     frac_of_burst=attn_tflops / peaks["bf16_burst"], frac_of_nominal=attn_tflops / 2250.0,
-                    launches_per_step=2, ms_per_step=float(np.mean(attn_ms)),
+                    launches_per_step=2 * n_layers, ms_per_step=float(np.mean(attn_ms)),
                     ms_global_pass=float(np.mean(attn_g_ms)),
                     traffic=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("bytes"),
                     traffic_note=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("source", "no ncu capture of this workload"),
@@ -417,24 +442,26 @@ def main():
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
+        run_layer(w, req)                      # leave layer 0's y in the buffer for the parity figure below
+        torch.cuda.synchronize()
         rows = pick_oracle_rows(w, args.oracle_pairs)
         dt, pairs, out = oracle_sample_run(w, rows)
-        allp = total_pairs(prof, req)
+        allp = total_pairs(prof, req)          # layer 0 (the layers have the same layout, own protected rows)
         # while the sample is at hand: parity of this very run against the checker
         from tests.helpers import rel_l2
         y_gpu = bufs["y"][torch.as_tensor(rows, device=dev)].float().cpu().numpy().astype(np.float64)
-        cpu_baseline = dict(value=req.T / (dt * allp / pairs), unit="tokens/s", cores=os.cpu_count(), kind="oracle",
+        cpu_baseline = dict(value=req.T / (dt * allp / pairs), unit="tokens/s (per layer)", cores=os.cpu_count(), kind="oracle",
                             threads=torch.get_num_threads(),
                             sample=f"{len(rows)} seeded rows, {pairs} of {allp} visible (row,key,head) pairs in "
                                    f"{dt:.1f} s, extrapolated by pair count",
                             pairs_per_s=pairs / dt, parity_rel_l2_y=rel_l2(y_gpu, out["y"]))
 
     line = dict(metric="mla_online_prefill_tokens_per_s_per_layer",
-                value=rkdist.aggregate_throughput(req.T, args.steps, world, total_ms_max * 1e-3),
+                value=rkdist.aggregate_throughput(req.T * n_layers, args.steps, world, total_ms_max * 1e-3),
                 unit="tokens/s", n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=total_ms_max / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="bf16", data="synthetic",
-                config=dict(workload=name, regime=args.regime, T=req.T, n_prot=req.A, n_segs=lay.n_segs,
+                config=dict(workload=name, regime=args.regime, layers=n_layers, T=req.T, n_prot=req.A, n_segs=lay.n_segs,
                             heads=prof.n_heads, groups=prof.n_groups, o_rank=prof.o_rank, d_model=prof.d_model,
                             l2="inputs larger than L2" if not need_flush else "L2 flushed between iterations",
                             flops_attn=fl_attn, flops_proj=fl_proj + fl_wb),
