@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -382,18 +383,33 @@ rk_status rk_request_create(rk_ctx* ctx, const rk_layout* lay, const int32_t* pr
       const double ang = (double)lay->seg_delta[i] * theta;
       cs[(size_t)i * 32 + j] = make_float2((float)std::cos(ang), (float)std::sin(ang));
     }
-  // visible-pair counts (for flop accounting): keys with pos <= row pos
-  auto visible = [&](int64_t pos) {
-    int64_t v = 0;
-    for (int i = 0; i < S; ++i) v += std::max<int64_t>(0, std::min<int64_t>(seg_n[(size_t)i], pos - seg_delta32[(size_t)i] + 1));
-    return v;
-  };
-  for (int64_t r = 0; r < T; ++r) rq->pairs_global += visible(row_pos[(size_t)r]);
+  // visible-pair counts (for flop accounting): a row of segment i at canonical index c sees every key
+  // of the segments placed before it in the request (intervals do not overlap) plus c + 1 of its own
+  std::vector<int64_t> keys_before((size_t)S, 0);
+  {
+    std::vector<int> order((size_t)S);
+    for (int i = 0; i < S; ++i) order[(size_t)i] = i;
+    std::sort(order.begin(), order.end(), [&](int a, int b) { return seg_delta32[(size_t)a] < seg_delta32[(size_t)b]; });
+    int64_t run = 0;
+    for (int k = 0; k < S; ++k) {
+      keys_before[(size_t)order[(size_t)k]] = run;
+      run += seg_n[(size_t)order[(size_t)k]];
+    }
+  }
+  for (int i = 0; i < S; ++i) {
+    const int64_t n = seg_n[(size_t)i];
+    rq->pairs_global += n * keys_before[(size_t)i] + n * (n + 1) / 2;
+  }
   std::vector<int32_t> prot((size_t)n_prot), prot_pos((size_t)n_prot);
-  for (int64_t a = 0; a < n_prot; ++a) {
-    prot[(size_t)a] = prot_rows[a];
-    prot_pos[(size_t)a] = row_pos[(size_t)prot_rows[a]];
-    rq->pairs_local += visible(prot_pos[(size_t)a]);
+  {
+    int seg = 0;
+    for (int64_t a = 0; a < n_prot; ++a) {
+      const int64_t r = prot_rows[a];
+      while (r >= lay->seg_off[seg + 1]) ++seg;  // the list is ascending
+      prot[(size_t)a] = (int32_t)r;
+      prot_pos[(size_t)a] = row_pos[(size_t)r];
+      rq->pairs_local += keys_before[(size_t)seg] + (r - lay->seg_off[seg]) + 1;
+    }
   }
   std::vector<AttnWorkItem> work_g, work_l;
   build_work(row_pos, ctx->prof.n_groups, seg_n, seg_delta32, ctx->n_pairs, &work_g);
@@ -480,6 +496,8 @@ static rk_status attn_pass(rk_ctx* ctx, const rk_request* rq, const void* kv, co
   AttnParams p;
   memset(&p, 0, sizeof(p));
   const int64_t n_flat = n_tok * hpt;
+  if (n_flat >= ((int64_t)1 << 31) - 256)
+    return fail(ctx, RK_ERR_LAYOUT, "rows x heads of one attention pass must stay below 2^31");
   rk_status s = make_tmap(ctx, &p.tm_q, q, (uint64_t)n_flat, kDQK, kDQK, 64, kAttnRowsPerCta);
   if (s != RK_OK) return s;
   s = make_tmap(ctx, &p.tm_kv, kv, (uint64_t)rq->T, kDQK, kDQK, 64, 128);
@@ -756,12 +774,14 @@ static __device__ __align__(256) unsigned char rk_static_scratch[RK_STATIC_SCRAT
 namespace {
 constexpr int kMaxDevices = 64;
 void* g_static_scratch_ptr[kMaxDevices] = {nullptr};
+std::mutex g_static_scratch_mutex;  // first calls may come from several host threads
 
 // Device address of rk_static_scratch on the CURRENT device (resolved once per device).  In host
 // code the array's name is only a handle for the runtime, not a device address, so the address
 // must come from cudaGetSymbolAddress.
 cudaError_t static_scratch_address(int device, void** out) {
   if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
   if (g_static_scratch_ptr[device] == nullptr) {
     void* ptr = nullptr;
     cudaError_t e = cudaGetSymbolAddress(&ptr, rk_static_scratch);

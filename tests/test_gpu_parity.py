@@ -410,3 +410,16 @@ def test_offline_then_online_chain_reuses_first_document_exactly(rk):
     assert_close(f64(y[lo:hi]), y_full[lo:hi], "first document rows vs full recomputation")
     inv = oracle.inverse_row_map(w.prot_rows, lay.n_rows)
     assert_close(f64(y)[inv >= 0], y_full[inv >= 0], "protected rows vs full recomputation")
+
+
+def test_request_info_pair_counts(rk):
+    """pairs_global / pairs_local (used for flop accounting) equal a brute-force count of visible keys."""
+    w = synth.make_custom([100, 260, 31], 20, n_heads=16, n_groups=2, o_rank=128, d_model=256, pct_bp=1000, seed=44)
+    lay = w.layout
+    lay.seg_delta = lay.seg_delta * 2 + 5             # gaps between segments
+    ctx, req = make(rk, w)
+    pos = oracle.request_positions(lay.seg_off, lay.seg_delta)
+    vis = (pos[None, :] <= pos[:, None]).sum(axis=1)
+    assert req.pairs_global == int(vis.sum())
+    assert req.pairs_local == int(vis[w.prot_rows].sum())
+    assert (req.T, req.A, req.n_off_rows) == (lay.n_rows, len(w.prot_rows), lay.n_doc_rows)
