@@ -372,7 +372,16 @@ def main():
         host = [(pin(wl.kv), pin(wl.q_g), pin(wl.q_l), pin(wl.z_off)) for wl, _ in layers]
         y_h = torch.empty((req.T, prof.d_model), dtype=torch.bfloat16).pin_memory()
 
+        if n_layers > 1:      # stack entry point: inputs of layer l+1 travel while layer l computes
+            bufs1 = ctx.alloc_layer_buffers(big, dev)
+            ys = [y_h] + [torch.empty_like(y_h).pin_memory() for _ in range(min(n_layers, 2) - 1)]
+            io = [dict(req=r, kv=h[0], q_g=h[1], q_l=h[2], z_off=h[3], W_uv=wl.w_uv, W_a=wl.w_a, W_b=wl.w_b,
+                       y=ys[i % len(ys)]) for i, ((wl, r), h) in enumerate(zip(layers, host))]
+
         def e2e_step():
+            if n_layers > 1:
+                rk.rk_layer_stack_host(ctx, io, bufs, bufs1)
+                return
             for (wl, r), (hk, hqg, hql, hzo) in zip(layers, host):
                 ctx.rk_layer_host(r, hk, hqg, hql, hzo, wl.w_uv, wl.w_a, wl.w_b, bufs, y_h)
 

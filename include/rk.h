@@ -231,6 +231,23 @@ rk_status rk_layer_host(rk_ctx* ctx, const rk_request* req, const void* kv_host,
                         const void* q_l_host, const void* z_off_host, const void* W_uv, const void* W_a,
                         const void* W_b, const rk_layer_buffers* dev, void* y_host, void* stream);
 
+/* One layer of a stack for rk_layer_stack_host. */
+typedef struct rk_layer_io {
+  const rk_request* req;                                    /* geometry + protected rows of this layer */
+  const void *kv_host, *q_g_host, *q_l_host, *z_off_host;   /* pinned host inputs (shapes as in rk_layer_host) */
+  const void *W_uv, *W_a, *W_b;                             /* device weights of this layer */
+  void* y_host;                                             /* pinned host output [T][d_model] */
+} rk_layer_io;
+
+/* A stack of layers from HOST inputs with cross-layer prefetch (Section "Turning omitted work into
+ * latency reduction": while layer l runs, a dedicated stream brings in the inputs of layer l+1;
+ * device events, not host polling, guard consumption).  Two complete buffer sets are used in turn:
+ * the inputs of layer l+1 are copied into the other set while layer l computes, and y of layer l
+ * is copied out on a third stream while layer l+1 computes.  Synchronises `stream` before it
+ * returns.  Every request must belong to `ctx`; the sets must be large enough for every layer. */
+rk_status rk_layer_stack_host(rk_ctx* ctx, int32_t n_layers, const rk_layer_io* layers, const rk_layer_buffers* dev0,
+                              const rk_layer_buffers* dev1, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -44,11 +44,16 @@ class rk_layer_buffers(C.Structure):
                                           "lse_g", "lse_l", "workspace")] + [("workspace_bytes", C.c_size_t)]
 
 
+class rk_layer_io(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("req", "kv_host", "q_g_host", "q_l_host", "z_off_host", "W_uv", "W_a", "W_b",
+                                          "y_host")]
+
+
 EXPORTS = ["rk_version", "rk_status_string", "rk_create", "rk_destroy", "rk_last_error", "rk_poll_status",
            "rk_set_wait_limit_ms", "rk_set_debug_flags", "rk_request_create", "rk_request_destroy", "rk_check_request",
            "rk_request_get_info", "rk_workspace_bytes", "rk_relocate_q", "rk_mla_online_attn",
            "rk_segmented_merge", "rk_group_sliced_proj", "rk_group_sliced_proj_static", "rk_combine_offline",
-           "rk_layer_host", "rk_mla_off_workspace_bytes", "rk_mla_off_build"]
+           "rk_layer_host", "rk_layer_stack_host", "rk_mla_off_workspace_bytes", "rk_mla_off_build"]
 
 
 def _load() -> C.CDLL:
@@ -80,6 +85,8 @@ def _load() -> C.CDLL:
     lib.rk_group_sliced_proj_static.argtypes = [vp] * 9
     lib.rk_combine_offline.argtypes = [vp] * 9
     lib.rk_layer_host.argtypes = [vp] * 9 + [C.POINTER(rk_layer_buffers), vp, vp]
+    lib.rk_layer_stack_host.argtypes = [vp, i32, C.POINTER(rk_layer_io), C.POINTER(rk_layer_buffers),
+                                        C.POINTER(rk_layer_buffers), vp]
     lib.rk_mla_off_workspace_bytes.argtypes = [vp, i64, C.POINTER(C.c_size_t)]
     lib.rk_mla_off_build.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp, vp, vp, C.c_size_t, vp]
     for name in EXPORTS:
@@ -275,6 +282,23 @@ class Context:
         self.check(lib.rk_layer_host(self.handle, req.handle, _ptr(kv_h), _ptr(q_g_h), _ptr(q_l_h), _ptr(z_off_h),
                                      _ptr(W_uv), _ptr(W_a), _ptr(W_b), C.byref(b), _ptr(y_h), _stream()))
         return y_h
+
+
+def _buffers_struct(bufs: dict) -> rk_layer_buffers:
+    return rk_layer_buffers(*[bufs[n].data_ptr() for n in ("kv", "q_g", "q_l", "z_off", "O_g", "O_l", "z_on_g", "z_on_l",
+                                                           "z", "y", "lse_g", "lse_l", "workspace")],
+                            bufs["workspace"].numel())
+
+
+def rk_layer_stack_host(ctx: "Context", layers, bufs0: dict, bufs1: dict):
+    """layers: list of dicts with keys req, kv, q_g, q_l, z_off (pinned host tensors), W_uv, W_a, W_b (device
+    tensors) and y (pinned host output).  Runs the stack with cross-layer prefetch."""
+    arr = (rk_layer_io * len(layers))()
+    for i, l in enumerate(layers):
+        arr[i] = rk_layer_io(l["req"].handle.value, _ptr(l["kv"]), _ptr(l["q_g"]), _ptr(l["q_l"]), _ptr(l["z_off"]),
+                             _ptr(l["W_uv"]), _ptr(l["W_a"]), _ptr(l["W_b"]), _ptr(l["y"]))
+    b0, b1 = _buffers_struct(bufs0), _buffers_struct(bufs1)
+    ctx.check(lib.rk_layer_stack_host(ctx.handle, len(layers), arr, C.byref(b0), C.byref(b1), _stream()))
 
 
 class Request:

@@ -35,6 +35,8 @@ struct rk_ctx {
   unsigned long long wait_ns = 2000ull * 1000 * 1000;
   int attn_debug = 0;  // development switches of the attention kernel (rk_set_debug_flags)
   cudaStream_t copy_stream = nullptr;  // rk_layer_host: copies that overlap the kernels
+  cudaStream_t copy_out_stream = nullptr;  // rk_layer_stack_host: device->host copies (full duplex with the above)
+  cudaEvent_t sev[6] = {nullptr};      // rk_layer_stack_host: in_ready[2], compute_done[2], y_copied[2]
   cudaEvent_t ev[8] = {nullptr};       // device-side ordering between the two streams (no host polling)
   PFN_encodeTiled encode = nullptr;
   mutable std::string err;
@@ -216,6 +218,8 @@ rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
   }
   ctx->n_pairs = attention_max_pairs(ctx->sm_count);
   e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_out_stream, cudaStreamNonBlocking);
+  for (int i = 0; i < 6 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->sev[i], cudaEventDisableTiming);
   for (int i = 0; i < 8 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -260,6 +264,9 @@ rk_status rk_destroy(rk_ctx* ctx) {
   for (int i = 0; i < 8; ++i)
     if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  for (int i = 0; i < 6; ++i)
+    if (ctx->sev[i]) cudaEventDestroy(ctx->sev[i]);
+  if (ctx->copy_out_stream) cudaStreamDestroy(ctx->copy_out_stream);
   cudaFree(ctx->d_status);
   cudaFree(ctx->d_batches);
   delete ctx;
@@ -754,6 +761,82 @@ rk_status rk_layer_host(rk_ctx* ctx, const rk_request* rq, const void* kv_host, 
   if (e == cudaSuccess) e = cudaStreamWaitEvent(st, ctx->ev[7], 0);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "device to host copy");
+}
+
+rk_status rk_layer_stack_host(rk_ctx* ctx, int32_t n_layers, const rk_layer_io* layers, const rk_layer_buffers* dev0,
+                              const rk_layer_buffers* dev1, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!layers || !dev0 || !dev1) return fail(ctx, RK_ERR_NULL, "null argument");
+  if (n_layers <= 0) return fail(ctx, RK_ERR_LAYOUT, "n_layers must be positive");
+  for (int l = 0; l < n_layers; ++l) {
+    const rk_layer_io& io = layers[l];
+    if (!io.req || !io.kv_host || !io.q_g_host || !io.W_uv || !io.W_a || !io.W_b || !io.y_host)
+      return fail(ctx, RK_ERR_NULL, "layer %d: null argument", l);
+    if (io.req->ctx != ctx) return fail(ctx, RK_ERR_LAYOUT, "layer %d: request belongs to another context", l);
+    if (io.req->A > 0 && !io.q_l_host) return fail(ctx, RK_ERR_NULL, "layer %d: q_l_host is required", l);
+    if (io.req->A < io.req->T && !io.z_off_host) return fail(ctx, RK_ERR_NULL, "layer %d: z_off_host is required", l);
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  cudaStream_t cin = ctx->copy_stream, cout = ctx->copy_out_stream;
+  cudaEvent_t* in_ready = ctx->sev;          // [2] inputs of buffer set b are on the device
+  cudaEvent_t* compute_done = ctx->sev + 2;  // [2] the layer running on set b has finished
+  cudaEvent_t* y_copied = ctx->sev + 4;      // [2] y of the layer that ran on set b is on the host
+  const rk_layer_buffers* sets[2] = {dev0, dev1};
+  const int G = ctx->prof.n_groups, L = ctx->prof.n_heads - G;
+  const size_t width = (size_t)G * ctx->prof.o_rank;
+
+  auto copy_in = [&](int l) -> cudaError_t {  // host -> device of layer l into set l & 1, on the copy-in stream
+    const rk_layer_io& io = layers[l];
+    const rk_request* rq = io.req;
+    const rk_layer_buffers* d = sets[l & 1];
+    cudaError_t e = cudaMemcpyAsync(d->kv, io.kv_host, (size_t)rq->T * kDQK * 2, cudaMemcpyHostToDevice, cin);
+    if (e == cudaSuccess && rq->A > 0)
+      e = cudaMemcpyAsync(d->q_l, io.q_l_host, (size_t)rq->A * L * kDQK * 2, cudaMemcpyHostToDevice, cin);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d->q_g, io.q_g_host, (size_t)rq->T * G * kDQK * 2, cudaMemcpyHostToDevice, cin);
+    if (e == cudaSuccess && rq->n_off_rows > 0 && io.z_off_host)
+      e = cudaMemcpyAsync(d->z_off, io.z_off_host, (size_t)rq->n_off_rows * width * 2, cudaMemcpyHostToDevice, cin);
+    if (e == cudaSuccess) e = cudaEventRecord(in_ready[l & 1], cin);
+    return e;
+  };
+
+  // everything already queued on `stream` comes first (the buffer sets may still be in use)
+  cudaError_t e = cudaEventRecord(ctx->ev[0], st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(cin, ctx->ev[0], 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(cout, ctx->ev[0], 0);
+  if (e == cudaSuccess) e = copy_in(0);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "host to device copy");
+  for (int l = 0; l < n_layers; ++l) {
+    const int b = l & 1;
+    const rk_layer_io& io = layers[l];
+    const rk_request* rq = io.req;
+    const rk_layer_buffers* d = sets[b];
+    const bool has_l = rq->A > 0;
+    if (l + 1 < n_layers) {  // prefetch the next layer while this one computes
+      if (l >= 1) e = cudaStreamWaitEvent(cin, compute_done[b ^ 1], 0);  // layer l-1 has released set b^1
+      if (e == cudaSuccess) e = copy_in(l + 1);
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "host to device copy");
+    }
+    e = cudaStreamWaitEvent(st, in_ready[b], 0);
+    if (e == cudaSuccess && l >= 2) e = cudaStreamWaitEvent(st, y_copied[b], 0);  // y of layer l-2 has left set b
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
+    rk_status s = rk_mla_online_attn(ctx, rq, d->kv, d->q_g, has_l ? d->q_l : nullptr, d->O_g, d->lse_g,
+                                     has_l ? d->O_l : nullptr, has_l ? d->lse_l : nullptr, stream);
+    if (s == RK_OK)
+      s = rk_group_sliced_proj(ctx, rq, d->O_g, has_l ? d->O_l : nullptr, io.W_uv, io.W_a, d->z_on_g,
+                               has_l ? d->z_on_l : nullptr, d->workspace, d->workspace_bytes, stream);
+    if (s == RK_OK) s = rk_combine_offline(ctx, rq, d->z_on_g, d->z_on_l, d->z_off, io.W_b, d->z, d->y, stream);
+    if (s != RK_OK) return s;
+    e = cudaEventRecord(compute_done[b], st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(cout, compute_done[b], 0);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(io.y_host, d->y, (size_t)rq->T * ctx->prof.d_model * 2, cudaMemcpyDeviceToHost, cout);
+    if (e == cudaSuccess) e = cudaEventRecord(y_copied[b], cout);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "device to host copy");
+  }
+  e = cudaStreamWaitEvent(st, y_copied[(n_layers - 1) & 1], 0);
+  if (e == cudaSuccess && n_layers >= 2) e = cudaStreamWaitEvent(st, y_copied[n_layers & 1], 0);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "stack synchronisation");
 }
 
 }  // extern "C"

@@ -423,3 +423,38 @@ def test_request_info_pair_counts(rk):
     assert req.pairs_global == int(vis.sum())
     assert req.pairs_local == int(vis[w.prot_rows].sum())
     assert (req.T, req.A, req.n_off_rows) == (lay.n_rows, len(w.prot_rows), lay.n_doc_rows)
+
+
+def test_layer_stack_host_matches_device_path(rk):
+    """Five independent layers (own values, own protected rows, shared layout) through the stack entry
+    point with cross-layer prefetch: every layer's y is bit-identical to the device-buffer path."""
+    layers, want = [], []
+    ctx = None
+    for l in range(5):
+        prof, lay, prot = synth.make_geometry("tiny", layer=l)
+        rng = np.random.default_rng(100 + l)
+        prot = synth.draw_protected_rows(lay, 300 + 200 * l, rng)            # a different row set per layer
+        w = synth.make_tensors("tiny", prof, lay, prot, 500 + l, regime="sharp")
+        if ctx is None:
+            ctx = rk.Context.from_profile(prof)
+        req = ctx.rk_request_create(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, prot)
+        pin = lambda t: t.cpu().pin_memory()
+        host = dict(req=req, kv=pin(w.kv), q_g=pin(w.q_g), q_l=pin(w.q_l), z_off=pin(w.z_off))
+        to_device(w)
+        O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
+        z_on_g, z_on_l = ctx.rk_group_sliced_proj(req, O_g, O_l, w.w_uv, w.w_a)
+        _, y = ctx.rk_combine_offline(req, z_on_g, z_on_l, w.z_off, w.w_b)
+        want.append(y.cpu())
+        host.update(W_uv=w.w_uv, W_a=w.w_a, W_b=w.w_b,
+                    y=torch.full((lay.n_rows, prof.d_model), float("nan"), dtype=torch.bfloat16).pin_memory())
+        layers.append(host)
+    ctx.rk_poll_status()
+    big = max(layers, key=lambda l: l["req"].A)["req"]
+    b0, b1 = ctx.alloc_layer_buffers(big, "cuda"), ctx.alloc_layer_buffers(big, "cuda")
+    for _ in range(2):                                     # twice: events and buffer sets are reused
+        rk.rk_layer_stack_host(ctx, layers, b0, b1)
+        ctx.rk_poll_status()
+        for l in range(5):
+            assert torch.equal(layers[l]["y"], want[l]), f"layer {l}"
+    rk.rk_layer_stack_host(ctx, layers[:1], b0, b1)         # a stack of one
+    assert torch.equal(layers[0]["y"], want[0])
