@@ -22,6 +22,12 @@
 #include "rk_internal.h"
 
 namespace rk {
+#ifdef RK_TRACE
+__device__ long long g_trace[4 * 16384];
+#define RK_TR(role, tag) do { if (blockIdx.x == 0 && lane == 0 && tr_n[role] < 8190) { g_trace[(role) * 16384 + 2 * tr_n[role]] = (tag); g_trace[(role) * 16384 + 2 * tr_n[role] + 1] = clock64(); ++tr_n[role]; } } while (0)
+#else
+#define RK_TR(role, tag) do { } while (0)
+#endif
 namespace {
 
 constexpr int kAttnThreads = 384;       // 4 role warps + 8 softmax warps
@@ -178,6 +184,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffAbort);
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + kOffTmemPtr);
   const uint64_t limit = p.wait_ns;
+#ifdef RK_TRACE
+  int tr_n[4] = {0, 0, 0, 0};
+#endif
 
   for (int i = threadIdx.x; i < 512; i += kAttnThreads) reinterpret_cast<volatile unsigned long long*>(smem + kOffXchg)[i] = 0ull;
   if (threadIdx.x == 0) {
@@ -233,6 +242,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         rp.advance();
         return true;
       }
+      RK_TR(2, 1);
       if (elect_one()) {
         const uint32_t full_local = bar(kBarRingFull + s);
         const uint32_t nbox = (col1 >= 0) ? 2u : 1u;
@@ -318,6 +328,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         int kt_pv = 0;      // key tiles whose PV has been issued
 
         auto issue_qk = [&](bool first_of_seg, bool last_of_seg, uint32_t rb) -> bool {
+          RK_TR(0, 1);
           if (first_of_seg) {
             if (!mbar_wait_bounded<true>(bar(kBarQrReady + rb), (qr_ready_phases >> rb) & 1u, limit, abort_flag,
                                          p.status, W_QRREADY, w))
@@ -331,6 +342,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             if (!mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
               return false;
             const uint32_t b_addr = smem_base + kOffRing + s * kStageBytes;
+            RK_TR(0, 10 + st);
             if (elect_one()) {
               if (st < 4) {
                 const uint32_t a_addr = q_base + 2 * st * kQChunkBytes;
@@ -359,6 +371,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             rp.advance();
           }
           ++kt_issued;
+          RK_TR(0, 2);
           return true;
         };
         auto issue_pv = [&]() -> bool {
@@ -366,6 +379,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             return false;
           p_ready_phase ^= 1;
           tc_fence_after_sync();
+          RK_TR(0, 3);
 #pragma unroll 1
           for (int q = 0; q < 4; ++q) {
             const int kh = q >> 1, h = q & 1;
@@ -374,6 +388,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
               return false;
             const uint32_t b_addr = smem_base + kOffRing + s * kStageBytes;
             const uint32_t tmem_o = tmem_base + kColO + (uint32_t)h * 128u;
+            RK_TR(0, 20 + q);
             if (elect_one()) {
               const uint64_t da = umma_desc_sw128(p_base + 2 * kh * kQChunkBytes, 16, 1024);
               const uint64_t db = umma_desc_sw128(b_addr, kChunkBytes, 1024);
@@ -389,6 +404,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             rp.advance();
           }
           ++kt_pv;
+          RK_TR(0, 4);
           return true;
         };
 
@@ -449,7 +465,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         }
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(mapa_shared(bar(kBarQrReady + rb), 0));
+        if (lane == 0) mbar_arrive_remote(mapa_shared(bar(kBarQrReady + rb), 0));
       }
     }
     // drain the last releases so that no commit targets this CTA after it exits
@@ -513,6 +529,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           s_full_phases ^= (1u << b);
           if (!ok) break;
           tc_fence_after_sync();
+          if (warp == 4) RK_TR(1, 1);
           if (p.debug & 1) {
             if (kt > 0) {
               ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
@@ -521,7 +538,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(p_ready_remote);
+            if (lane == 0) mbar_arrive_remote(p_ready_remote);
             continue;
           }
           uint32_t s[64];
@@ -542,6 +559,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           float mxo = mx;
           if (!(p.debug & 4)) ok = quad_exchange_max(xbuf, part, m, ++xseq, mx, mxo, limit, abort_flag, p.status, w);
           if (!ok) break;
+          if (warp == 4) RK_TR(1, 2);
           const float mt = mxo * scale;
           // lazy rescale: only when the running maximum grows by more than 2^8
           float alpha = 1.f;
@@ -573,12 +591,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             }
           }
           l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+          if (warp == 4) RK_TR(1, 3);
           // P buffer and O are free once the previous PV has completed
           if (kt > 0) {
             ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
             pv_done_phase ^= 1;
             if (!ok) break;
             tc_fence_after_sync();
+            if (warp == 4) RK_TR(1, 4);
             if (__any_sync(0xffffffffu, need)) {
 #pragma unroll 1
               for (int cc = 0; cc < 128; cc += 32) {  // this thread's 2 x 64 columns of O
@@ -603,7 +623,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           fence_proxy_async_smem();
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(p_ready_remote);
+          if (lane == 0) mbar_arrive_remote(p_ready_remote);
+          if (warp == 4) RK_TR(1, 5);
         }
       }
       if (!ok) break;
@@ -658,6 +679,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     tmem_dealloc<2>(tmem_base, 512);
   }
 }
+
+#ifdef RK_TRACE
+extern "C" int rk_debug_read_trace(long long* out, int n) {
+  return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * (size_t)n);
+}
+#endif
 
 cudaError_t attention_setup() {
   return cudaFuncSetAttribute(rk_mla_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);

@@ -64,9 +64,17 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// arrive on a barrier that lives in another CTA of the cluster (address from mapa)
+// arrive on a barrier that lives in another CTA of the cluster (address from mapa), with a
+// cluster-scope release: everything this thread wrote becomes visible cluster-wide first (slow)
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// the same arrive with the default (CTA-scope) release: enough when the data the arrival announces
+// was written to this CTA's own shared memory and published to the async proxy by
+// fence.proxy.async -- the waiting thread in the peer CTA only issues the MMA, this CTA's tensor
+// core reads the data
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
