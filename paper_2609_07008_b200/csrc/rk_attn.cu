@@ -9,14 +9,22 @@
 //   S[64 x 256 keys]  = Q[64 x 576] K^T         9 k-chunks of 64 (8 latent, then the rotated rope)
 //   O[64 x 512]      += P[64 x 256] V[256 x 512] two N=256 halves
 // In that UMMA shape each CTA's 64 accumulator rows fold onto all 128 TMEM lanes (lanes 0-63:
-// columns [0,N/2), lanes 64-127: columns [N/2,N)), so O takes 256 columns and two S buffers
-// 2 x 128: exactly the 512 columns of TMEM.  The B operand is split across the pair: for QK^T
-// each CTA streams its 128 keys of the tile, for PV its 128 of each 256 output dims.  The same
-// [128 keys x 64 dims] 128B-swizzled TMA box serves as K-major B (QK^T) and MN-major B (PV).
+// columns [0,N/2), lanes 64-127: columns [N/2,N)), so O takes 256 columns and the score buffer S
+// 128.  The remaining 128 columns hold latent dims 256-511 of the Q tile (bf16 pairs, the rows in
+// both lane halves) and feed the QK^T MMAs of those dims as a tensor-memory A operand; only dims
+// 0-255 and the rope chunk of Q stay in shared memory.  The 32 KB that frees pay for a fourth
+// 32 KB stage of the K/V ring, which is what keeps the tensor pipe fed while the per-SM L2 -> SMEM
+// rate (about 76 B/clk) trails the MMA's appetite within a tile.  S is single-buffered: QK^T of
+// the next key tile follows the PV of the previous one in the issue order, and by then the
+// softmax warps have long read S into registers (the s_free barrier states it).
+// The B operand is split across the pair: for QK^T each CTA streams its 128 keys of the tile,
+// for PV its 128 of each 256 output dims.  The same [128 keys x 64 dims] 128B-swizzled TMA box
+// serves as K-major B (QK^T) and MN-major B (PV).
 //
 // Warp roles per CTA (384 threads): warp 0 TMA producer, warp 1 UMMA issuer (leader CTA only),
 // warp 2 query relocation, warps 4-11 softmax / correction / epilogue (two warps per TMEM lane
-// quarter, each owning half of the columns).
+// quarter, each owning half of the columns).  At the start of a row tile the upper Q half lands
+// in one ring stage and the softmax warps copy it into TMEM (tcgen05.st) before their first scores.
 #include <cuda_bf16.h>
 
 #include "rk_internal.h"
@@ -31,22 +39,23 @@ __device__ long long g_trace[4 * 16384];
 namespace {
 
 constexpr int kAttnThreads = 384;       // 4 role warps + 8 softmax warps
-constexpr int kStages = 3;                // ring of 32 KB stages (two 16 KB TMA boxes each)
+constexpr int kStages = 4;                // ring of 32 KB stages (two 16 KB TMA boxes each)
 constexpr uint32_t kChunkBytes = 16384;  // 128 keys x 64 dims bf16
 constexpr uint32_t kStageBytes = 2 * kChunkBytes;
 constexpr uint32_t kQChunkBytes = 8192;  // 64 rows x 64 dims bf16
 
 // shared memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t kOffQLat = 0;                                // 8 chunks
-constexpr uint32_t kOffQPristine = kOffQLat + 8 * kQChunkBytes;  // rope chunk as loaded
+constexpr uint32_t kOffQLat = 0;                                // latent dims 0-255: 4 chunks (dims 256-511 live in TMEM)
+constexpr uint32_t kOffQPristine = kOffQLat + 4 * kQChunkBytes;  // rope chunk as loaded
 constexpr uint32_t kOffQRot = kOffQPristine + kQChunkBytes;      // 2 rotated rope chunks
 constexpr uint32_t kOffP = kOffQRot + 2 * kQChunkBytes;          // 4 sub-chunks [64 x 64 keys]
 constexpr uint32_t kOffRing = kOffP + 4 * kQChunkBytes;
 constexpr uint32_t kOffBars = kOffRing + kStages * kStageBytes;
 // barrier indices (8 bytes each)
 constexpr int kBarQFull = 0, kBarQFree = 1, kBarQrReady = 2 /*2*/, kBarQrFree = 4 /*2*/, kBarRingFull = 6,
-              kBarRingEmpty = kBarRingFull + kStages, kBarSFull = kBarRingEmpty + kStages /*2*/,
-              kBarPReady = kBarSFull + 2, kBarPvDone = kBarPReady + 1, kNumBars = kBarPvDone + 1;
+              kBarRingEmpty = kBarRingFull + kStages, kBarSFull = kBarRingEmpty + kStages,
+              kBarSFree = kBarSFull + 1, kBarPReady = kBarSFree + 1, kBarPvDone = kBarPReady + 1,
+              kBarQhFull = kBarPvDone + 1, kBarQhDone = kBarQhFull + 1, kNumBars = kBarQhDone + 1;
 constexpr uint32_t kOffTmemPtr = kOffBars + kNumBars * 8;
 constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
 constexpr uint32_t kOffXchg = kOffAbort + 8;                 // u64 [2 parity][4 parts][64]: (seq << 32) | value
@@ -55,13 +64,14 @@ constexpr uint32_t kSmemBytes = kSmemUsed + 1024;            // + alignment slac
 
 // TMEM columns
 constexpr uint32_t kColO = 0;    // two halves of 128 columns
-constexpr uint32_t kColS = 256;  // two buffers of 128 columns
+constexpr uint32_t kColS = 256;  // one 128-column score buffer
+constexpr uint32_t kColQ = 384;  // latent dims 256-511 of the Q tile as a TMEM A operand (both lane halves hold the rows)
 
 constexpr uint32_t kIdescQK = umma_idesc_bf16(128, 256, 0, 0);
 constexpr uint32_t kIdescPV = umma_idesc_bf16(128, 256, 0, 1);
 
 // wait tags reported on timeout
-enum { W_QFULL = 1, W_QFREE, W_QRREADY, W_QRFREE, W_RINGFULL, W_RINGEMPTY, W_SFULL, W_PREADY, W_PVDONE, W_DRAIN };
+enum { W_QFULL = 1, W_QFREE, W_QRREADY, W_QRFREE, W_RINGFULL, W_RINGEMPTY, W_SFULL, W_PREADY, W_PVDONE, W_DRAIN, W_SFREE, W_QHFULL, W_QHDONE };
 
 struct SegIter {
   // Iterates the segments a row tile can see; kmax = number of canonical keys of the segment that
@@ -196,8 +206,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar(kBarQrReady + b), 2);
       mbar_init(bar(kBarQrFree + b), 1);
-      mbar_init(bar(kBarSFull + b), 1);
     }
+    mbar_init(bar(kBarSFull), 1);
+    mbar_init(bar(kBarSFree), 16);   // every softmax warp of the pair has read the score buffer
+    mbar_init(bar(kBarQhFull), 1);   // this CTA's upper Q half has landed in its ring stage
+    mbar_init(bar(kBarQhDone), 16);  // every softmax warp of the pair has moved its part into TMEM
     for (int s = 0; s < kStages; ++s) {
       mbar_init(bar(kBarRingFull + s), 1);
       mbar_init(bar(kBarRingEmpty + s), 1);
@@ -278,13 +291,34 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         qfree_phase ^= 1;
         if (!ok) break;
       }
-      if (elect_one()) {
-        mbar_arrive_expect_tx(bar(kBarQFull), 9 * kQChunkBytes);
-        const int qrow = item.tile * kAttnRowsPerPair + (int)crank * kAttnRowsPerCta;
-        for (int d = 0; d < 9; ++d)
+      const int qrow = item.tile * kAttnRowsPerPair + (int)crank * kAttnRowsPerCta;
+      if (elect_one()) {  // lower latent half and the rope chunk stay in shared memory for the whole row tile
+        mbar_arrive_expect_tx(bar(kBarQFull), 5 * kQChunkBytes);
+        for (int d = 0; d < 4; ++d)
           tma_load_2d_hint(smem_base + kOffQLat + d * kQChunkBytes, &p.tm_q, bar(kBarQFull), d * 64, qrow, pol_q);
+        tma_load_2d_hint(smem_base + kOffQPristine, &p.tm_q, bar(kBarQFull), kDLatent, qrow, pol_q);
       }
       __syncwarp();
+      // Upper latent half (dims 256-511): staged through one ring stage, from where the softmax warps move
+      // it into tensor memory.  Each CTA loads its own rows and signals its own barrier; the issuer lets go
+      // of the ring position once both CTAs have finished the move.
+      {
+        const uint32_t s = rp.stage();
+        if (rp.it >= (uint32_t)kStages) {
+          ok = mbar_wait_bounded<false>(bar(kBarRingEmpty + s), rp.parity() ^ 1u, limit, abort_flag, p.status,
+                                        W_RINGEMPTY, w);
+          if (!ok) break;
+        }
+        if (!(p.debug & 8) && elect_one()) {
+          if (leader) mbar_arrive(bar(kBarRingFull + s));  // keeps the ring's phases in step; no bytes land here
+          mbar_arrive_expect_tx(bar(kBarQhFull), 4 * kQChunkBytes);
+          for (int d = 0; d < 4; ++d)
+            tma_load_2d_hint(smem_base + kOffRing + s * kStageBytes + d * kQChunkBytes, &p.tm_q, bar(kBarQhFull),
+                             256 + d * 64, qrow, pol_q);
+        }
+        __syncwarp();
+        rp.advance();
+      }
       // order of consumption: K(0), K(1), V(0), K(2), V(1), ..., V(last)
       SegIter it(p, item);
       int prev_row0 = -1, prev_kb = 0;
@@ -316,6 +350,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       RingPos rp;
       uint32_t qr_ready_phases = 0;  // bit rb = parity to wait for
       uint32_t p_ready_phase = 0;
+      uint32_t qh_done_phase = 0;
+      uint32_t s_writes = 0;  // how often the score buffer has been written (gives the s_free phase)
       uint32_t qr_use = 0;  // counts rope-buffer uses across tiles
       bool ok = true;
       const uint32_t q_base = smem_base + kOffQLat;
@@ -326,6 +362,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         const int n_kt = count_key_tiles(p, item);
         int kt_issued = 0;  // key tiles whose QK^T has been issued
         int kt_pv = 0;      // key tiles whose PV has been issued
+        {  // ring position of the staged upper Q half: wait for both CTAs' move into TMEM, then let go of it
+          const uint32_t s = rp.stage();
+          ok = mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w) &&
+               mbar_wait_bounded<true>(bar(kBarQhDone), qh_done_phase, limit, abort_flag, p.status, W_QHDONE, w);
+          qh_done_phase ^= 1;
+          if (!ok) break;
+          tc_fence_after_sync();
+          if (elect_one()) umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
+          __syncwarp();
+          rp.advance();
+        }
 
         auto issue_qk = [&](bool first_of_seg, bool last_of_seg, uint32_t rb) -> bool {
           RK_TR(0, 1);
@@ -335,7 +382,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
               return false;
             qr_ready_phases ^= (1u << rb);
           }
-          const uint32_t tmem_s = tmem_base + kColS + (uint32_t)(kt_issued & 1) * 128u;
+          if (s_writes > 0) {  // one score buffer: the softmax warps must have read the previous key tile's scores
+            if (!mbar_wait_bounded<true>(bar(kBarSFree), (s_writes - 1) & 1u, limit, abort_flag, p.status, W_SFREE, w))
+              return false;
+            tc_fence_after_sync();
+          }
+          ++s_writes;
+          const uint32_t tmem_s = tmem_base + kColS;
 #pragma unroll 1
           for (int st = 0; st < 5; ++st) {
             const uint32_t s = rp.stage();
@@ -344,7 +397,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             const uint32_t b_addr = smem_base + kOffRing + s * kStageBytes;
             RK_TR(0, 10 + st);
             if (elect_one()) {
-              if (st < 4) {
+              if (st >= 2 && st < 4) {  // latent dims 256-511: A from tensor memory, 8 columns per K = 16 step
+                const uint32_t a_tmem = tmem_base + kColQ + (uint32_t)(st - 2) * 64u;
+                const uint64_t db = umma_desc_sw128(b_addr, 16, 1024);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                  umma_f16_ts<2>(tmem_s, a_tmem + 8u * k, db + (uint64_t)(((k >> 2) * kChunkBytes + (k & 3) * 32) >> 4),
+                                 kIdescQK, 1u);
+                }
+                umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
+              } else if (st < 2) {  // latent dims 0-255: A from shared memory
                 const uint32_t a_addr = q_base + 2 * st * kQChunkBytes;
                 // descriptors differ only in the start-address field (16-byte units): add constants
                 const uint64_t da = umma_desc_sw128(a_addr, 16, 1024), db = umma_desc_sw128(b_addr, 16, 1024);
@@ -361,7 +423,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
 #pragma unroll
                 for (int k = 0; k < 4; ++k) umma_f16<2>(tmem_s, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), kIdescQK, 1u);
                 umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
-                umma_commit_2_mc(bar(kBarSFull + (kt_issued & 1)), 3);
+                umma_commit_2_mc(bar(kBarSFull), 3);
                 if (last_of_seg) umma_commit_2_mc(bar(kBarQrFree + rb), 3);
                 // all QK^T of this row tile issued: the Q tile is free once they complete
                 if (kt_issued + 1 == n_kt) umma_commit_2_mc(bar(kBarQFree), 3);
@@ -491,11 +553,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     const uint32_t lane_base = ((uint32_t)((sw & 3) * 32)) << 16;
     volatile unsigned long long* xbuf = reinterpret_cast<volatile unsigned long long*>(smem + kOffXchg);
     uint32_t xseq = 0;  // exchange sequence number
-    uint32_t s_full_phases = 0;  // bit b = parity to wait for
+    uint32_t ring_it = 0;  // ring position of the current row tile's staged Q half
+    uint32_t s_full_phase = 0;
+    uint32_t qh_full_phase = 0;
     uint32_t pv_done_phase = 0;
     bool ok = true;
     const float scale = p.scale_log2;
     const uint32_t p_ready_remote = mapa_shared(bar(kBarPReady), 0);
+    const uint32_t s_free_remote = mapa_shared(bar(kBarSFree), 0);
+    const uint32_t qh_done_remote = mapa_shared(bar(kBarQhDone), 0);
 
     for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
       const AttnWorkItem item = get_work(p, w);
@@ -509,6 +575,29 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       }
       float m_run = -INFINITY, l_run = 0.f;
       int kt = 0;
+      {  // move this thread's share of the upper Q half (row m, 64 dims) from its ring stage into TMEM
+        ok = mbar_wait_bounded<false>(bar(kBarQhFull), qh_full_phase, limit, abort_flag, p.status, W_QHFULL, w);
+        qh_full_phase ^= 1;
+        if (!ok) break;
+        // every role counts ring positions alike: one staged half per row tile, nine stages per key tile
+        const uint8_t* stage = smem + kOffRing + (ring_it % kStages) * kStageBytes;
+        ring_it += 1u + 9u * (uint32_t)count_key_tiles(p, item);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t qv[32];
+          const uint8_t* chunk = stage + (2 * ch + half) * kQChunkBytes;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint4 v = *reinterpret_cast<const uint4*>(chunk + sw128_offset((uint32_t)m, (uint32_t)c));
+            qv[4 * c] = v.x; qv[4 * c + 1] = v.y; qv[4 * c + 2] = v.z; qv[4 * c + 3] = v.w;
+          }
+          tmem_st_x32(tmem_base + lane_base + kColQ + (uint32_t)(ch * 64 + half * 32), qv);
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_remote(qh_done_remote);
+      }
 
       SegIter it(p, item);
       while (ok && it.next()) {
@@ -523,14 +612,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         for (int kb = 0; kb < it.kmax && ok; kb += kAttnKeysPerTile, ++kt) {
           int nv = lim - (kb + part * 64) + 1;
           nv = nv < 0 ? 0 : (nv > 64 ? 64 : nv);
-          const int b = kt & 1;
-          ok = mbar_wait_bounded<false>(bar(kBarSFull + b), (s_full_phases >> b) & 1u, limit, abort_flag, p.status,
-                                        W_SFULL, w);
-          s_full_phases ^= (1u << b);
+          ok = mbar_wait_bounded<false>(bar(kBarSFull), s_full_phase, limit, abort_flag, p.status, W_SFULL, w);
+          s_full_phase ^= 1;
           if (!ok) break;
           tc_fence_after_sync();
           if (warp == 4) RK_TR(1, 1);
           if (p.debug & 1) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(s_free_remote);
             if (kt > 0) {
               ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
               pv_done_phase ^= 1;
@@ -542,10 +631,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             continue;
           }
           uint32_t s[64];
-          const uint32_t taddr = tmem_base + lane_base + kColS + (uint32_t)b * 128u + (uint32_t)ch * 64u;
+          const uint32_t taddr = tmem_base + lane_base + kColS + (uint32_t)ch * 64u;
           tmem_ld_x32(taddr + 0, s + 0);
           tmem_ld_x32(taddr + 32, s + 32);
           tmem_wait_ld();
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_remote(s_free_remote);  // the issuer may overwrite the score buffer
           const bool full = __all_sync(0xffffffffu, nv == 64);  // no masking needed anywhere in this warp
           float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
           if (full) {
