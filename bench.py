@@ -34,9 +34,9 @@ FLOP_PER_PAIR = 2 * 576 + 2 * 512     # QK^T over 576 + PV over 512 per visible 
 # dram__bytes_read.sum + dram__bytes_write.sum of the attention kernel's two launches per step, from the
 # one-pass ncu captures summarised under profiles/ (bytes per step; None where no capture exists)
 PROFILED_DRAM_TRAFFIC = {
-    "flash256k": dict(bytes=37.80e9 + 9.22e9, algorithmic=4.91e9 + 1.20e9,
+    "flash256k": dict(bytes=37.44e9 + 9.58e9, algorithmic=4.91e9 + 1.20e9,
                       source="profiles/attn_kernel_flash256k_dram_traffic.md"),
-    "flash1": dict(bytes=(355.0e6 + 234.6e6) + (180.5e6 + 84.0e6), algorithmic=(350.3e6 + 277.9e6) + (168.4e6 + 115.5e6),
+    "flash1": dict(bytes=(352.0e6 + 224.9e6) + (169.6e6 + 74.8e6), algorithmic=(350.3e6 + 277.9e6) + (168.4e6 + 115.5e6),
                    source="profiles/attn_kernel_flash1_ncu_full.md"),
 }
 L2_BYTES = 126 * 1024 * 1024
