@@ -19,3 +19,4 @@ artifacts is from full recomputation on random data) -- the paper quantifies tha
 through model-level F1/EM, so there is nothing to pin it to.
 """
 from .mla_online import *  # noqa: F401,F403
+from . import policy  # noqa: F401  (Eq. protected and Eq. moe; pins in tests/test_oracle_policy_pins.py)
