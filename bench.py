@@ -223,6 +223,47 @@ def time_stream_kernels(ctx, req, w, prof, lay, dev, budget_bytes=6 << 30):
     return res
 
 
+def time_selection_rules(ctx, lay, dev):
+    """rk_protected_rows on the bench request with the paper's constants at the 25 % budget (flag pass,
+    8 select passes, 3 compaction passes; the time is launch latency, the bytes are a few per row) and
+    rk_moe_fanout on 16 M tokens (26 B per token, a plain streaming pass)."""
+    from paper_2609_07008_b200 import synth as _synth
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, reps=10):
+        for _ in range(3):
+            fn()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, b in evs:
+            a.record(stream)
+            fn()
+            b.record(stream)
+        torch.cuda.synchronize()
+        return float(np.mean([a.elapsed_time(b) for a, b in evs]))
+
+    res = {}
+    dirty, scores = _synth.draw_policy_inputs(lay, seed=99, n_dirty=500)
+    d, s = torch.from_numpy(dirty).to(dev), torch.from_numpy(scores).to(dev)
+    T, S = lay.n_rows, lay.n_segs
+    out = ctx.rk_protected_rows(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, d, s, budget_bp=2500)
+    ws = torch.empty(16 << 20, dtype=torch.uint8, device=dev)
+    ms = timed(lambda: ctx.rk_protected_rows(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, d, s, budget_bp=2500,
+                                             out=out, workspace=ws))
+    n_sel = int(out[1].item())
+    # per row: flag pass 1 B written; 8 select passes 1 B flag + 4 B score; count 5 B; scatter 5 B + output
+    nbytes = T * (1 + 8 * 5 + 5 + 5) + 4 * n_sel + 4 * len(dirty)
+    res["rk_protected_rows"] = dict(ms=ms, rows=T, selected=n_sel, budget_bp=2500, launches=13, bytes=nbytes,
+                                    gbs=nbytes / ms / 1e6, bound="launch latency (13 short kernels + 4 small copies)")
+    n = 16 << 20
+    p = torch.rand((n, 6), device=dev, dtype=torch.float32) + 0.01
+    k, keep = ctx.rk_moe_fanout(p, 0.85)
+    ms = timed(lambda: ctx.rk_moe_fanout(p, 0.85, False, k, keep))
+    nbytes = n * 26
+    res["rk_moe_fanout"] = dict(ms=ms, tokens=n, bytes=nbytes, gbs=nbytes / ms / 1e6)
+    ctx.rk_poll_status()
+    return res
+
+
 def time_offline_build(ctx, req, w, prof, lay, dev, rows_per_call=65536):
     """Offline MLA-Off artifact build (Algorithm 1) over every document row, in row ranges; not part of
     the online step.  Flops: 2176 per visible (row, key, Local head) pair inside each document alone,
@@ -404,6 +445,7 @@ def main():
     aux = None
     if not args.no_aux and rank == 0:
         aux = time_stream_kernels(ctx, req, w, prof, lay, dev)
+        aux.update(time_selection_rules(ctx, lay, dev))
 
     # where the rest of the step goes (instrumentation pass, not the timed region)
     breakdown = None

@@ -211,6 +211,56 @@ rk_status rk_mla_off_build(rk_ctx* ctx, const rk_request* req, const void* kv, i
                            const void* q_l_rows, const void* W_uv, const void* W_a, void* z_off_rows, void* workspace,
                            size_t workspace_bytes, void* stream);
 
+/* Controller of the protected-row set (Eq. protected).  The paper's values: edge_rows 128,
+ * tail_rows 32768, budget_bp 0 (no expansion), 1000, 2000 or 2500. */
+typedef struct rk_policy {
+  int32_t edge_rows;  /* B_edge: first and last rows of every relocated segment; >= 0 */
+  int64_t tail_rows;  /* T_tail: the last request positions; >= 0 */
+  int32_t budget_bp;  /* active budget in basis points of the candidate rows; 0..10000 */
+} rk_policy;
+
+/* Builds the protected token-row set A = Q u N u D u B_edge u I_top u T_tail (Eq. protected;
+ * `ProtectedRows` of Algorithm 2) on the device, as the strictly ascending packed-row list that
+ * rk_request_create takes.  Packed row t of segment i has canonical index j = t - seg_off[i] and
+ * request position seg_delta[i] + j.
+ *   Q u N   every row of a segment without artifact
+ *   D       dirty_rows: device int32 [n_dirty], any order, duplicates allowed, entries outside
+ *           [0,T) ignored; may be NULL iff n_dirty == 0
+ *   B_edge  rows with j < edge_rows or j >= n_i - edge_rows of every segment that has an artifact
+ *           and seg_delta[i] != 0 (artifacts are built at offset 0; any other offset relocates)
+ *   T_tail  rows at request positions >= end - tail_rows, end = largest position + 1
+ *   I_top   candidate rows = rows of segments with artifact.  If the sets above hold fewer than
+ *           floor(budget_bp * candidates / 10000) candidate rows, the candidate rows outside them
+ *           with the largest scores are added until that number is reached (equal scores: lower
+ *           packed row first; -0.0 equals +0.0).  The sets above are never cut.
+ *           scores: device float32 [T] (the Indexer's row scores, recomputed by the caller for
+ *           this request; entries of non-candidate rows are not read), no NaN; NULL = no top-up.
+ *   rows_out  device int32 [T] (capacity); the first *count_out entries are the result
+ *   count_out device int64 [1]
+ *   workspace device scratch of at least rk_protected_rows_workspace_bytes(T, n_segs), 256-byte aligned
+ * The layout is host data and is validated like in rk_request_create (RK_ERR_LAYOUT).  The call
+ * enqueues on `stream` and does not synchronise; read rows_out / count_out after the stream has
+ * passed it.  The selection is exact (integer work; the scores are only compared), so the list is
+ * bit-identical to the definition. */
+rk_status rk_protected_rows_workspace_bytes(int64_t n_rows, int32_t n_segs, size_t* out);
+rk_status rk_protected_rows(rk_ctx* ctx, const rk_layout* layout, const rk_policy* policy, const int32_t* dirty_rows,
+                            int64_t n_dirty, const float* scores, int32_t* rows_out, int64_t* count_out,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/* Retained expert fan-out of the adaptive sparse-MoE path (Eq. moe) for n tokens.
+ *   p        device float32 [n][6]: the router weights of the token's Top-6 experts, any slot
+ *            order, positive, no NaN; 8-byte aligned
+ *   tau      the cumulative-share threshold
+ *   fence    non-zero: a full-recompute fence layer, every token keeps all six (K_t = 6)
+ *   k_out    device uint8 [n]: K_t in {3,4,5,6}
+ *   keep_out device uint8 [n]: bit s set = the expert in slot s stays (the K_t largest weights;
+ *            equal weights: lower slot first)
+ * The weights are not renormalised and not written.  Decision arithmetic (float32, fixed order):
+ * weights sorted descending, c_1 = p_(1), c_k = c_(k-1) + p_(k); K_t = the smallest k in {3,4,5}
+ * with c_k >= tau * c_6, else 6 -- the paper's condition with both sides multiplied by the sum. */
+rk_status rk_moe_fanout(rk_ctx* ctx, const float* p, int64_t n, float tau, int32_t fence, uint8_t* k_out,
+                        uint8_t* keep_out, void* stream);
+
 /* Device buffers that rk_layer_host stages through; all owned by the caller. */
 typedef struct rk_layer_buffers {
   void *kv, *q_g, *q_l, *z_off;            /* device copies of the per-request inputs */

@@ -33,6 +33,10 @@ class rk_layout(C.Structure):
                 ("seg_has_artifact", C.POINTER(C.c_uint8))]
 
 
+class rk_policy(C.Structure):
+    _fields_ = [("edge_rows", C.c_int32), ("tail_rows", C.c_int64), ("budget_bp", C.c_int32)]
+
+
 class rk_request_info(C.Structure):
     _fields_ = [("n_rows", C.c_int64), ("n_prot", C.c_int64), ("n_off_rows", C.c_int64),
                 ("pairs_global", C.c_int64), ("pairs_local", C.c_int64), ("n_tiles_global", C.c_int32),
@@ -53,7 +57,8 @@ EXPORTS = ["rk_version", "rk_status_string", "rk_create", "rk_destroy", "rk_last
            "rk_set_wait_limit_ms", "rk_set_debug_flags", "rk_request_create", "rk_request_destroy", "rk_check_request",
            "rk_request_get_info", "rk_workspace_bytes", "rk_relocate_q", "rk_mla_online_attn",
            "rk_segmented_merge", "rk_group_sliced_proj", "rk_group_sliced_proj_static", "rk_combine_offline",
-           "rk_layer_host", "rk_layer_stack_host", "rk_mla_off_workspace_bytes", "rk_mla_off_build"]
+           "rk_layer_host", "rk_layer_stack_host", "rk_mla_off_workspace_bytes", "rk_mla_off_build",
+           "rk_protected_rows_workspace_bytes", "rk_protected_rows", "rk_moe_fanout"]
 
 
 def _load() -> C.CDLL:
@@ -89,6 +94,10 @@ def _load() -> C.CDLL:
                                         C.POINTER(rk_layer_buffers), vp]
     lib.rk_mla_off_workspace_bytes.argtypes = [vp, i64, C.POINTER(C.c_size_t)]
     lib.rk_mla_off_build.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp, vp, vp, C.c_size_t, vp]
+    lib.rk_protected_rows_workspace_bytes.argtypes = [i64, i32, C.POINTER(C.c_size_t)]
+    lib.rk_protected_rows.argtypes = [vp, C.POINTER(rk_layout), C.POINTER(rk_policy), vp, i64, vp, vp, vp, vp,
+                                      C.c_size_t, vp]
+    lib.rk_moe_fanout.argtypes = [vp, vp, i64, C.c_float, i32, vp, vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is C.c_int:  # default restype: rk_status
@@ -238,6 +247,43 @@ class Context:
         self.check(lib.rk_group_sliced_proj_static(self.handle, req.handle, _ptr(O_g), _ptr(O_l), _ptr(W_uv),
                                                    _ptr(W_a), _ptr(z_on_g), _ptr(z_on_l), _stream()))
         return z_on_g, z_on_l
+
+    def rk_protected_rows(self, seg_off, seg_delta, seg_has_artifact, dirty_rows=None, scores=None, *, edge_rows=128,
+                          tail_rows=32768, budget_bp=0, device="cuda", out=None, workspace=None):
+        """Eq. (protected) on the device.  Returns (rows_out, count_out): a device int32 buffer of capacity T
+        whose first count_out[0] entries are the ascending protected rows, and the device int64 count.
+        Nothing is synchronised; `protected_rows_to_host` reads the list back."""
+        lay, keep = make_layout_struct(seg_off, seg_delta, seg_has_artifact)
+        pol = rk_policy(int(edge_rows), int(tail_rows), int(budget_bp))
+        T, S = int(keep[0][-1]), len(keep[1])
+        if workspace is None:
+            need = C.c_size_t(0)
+            s = lib.rk_protected_rows_workspace_bytes(T, S, C.byref(need))
+            if s != 0:
+                raise RKError(s, "rk_protected_rows_workspace_bytes")
+            workspace = torch.empty(need.value, dtype=torch.uint8, device=device)
+        if out is None:
+            out = (torch.empty(T, dtype=torch.int32, device=device), torch.empty(1, dtype=torch.int64, device=device))
+        n_dirty = 0 if dirty_rows is None else dirty_rows.numel()
+        self.check(lib.rk_protected_rows(self.handle, C.byref(lay), C.byref(pol), _ptr(dirty_rows), n_dirty, _ptr(scores),
+                                         _ptr(out[0]), _ptr(out[1]), _ptr(workspace), workspace.numel(), _stream()))
+        return out
+
+    @staticmethod
+    def protected_rows_to_host(out) -> np.ndarray:
+        n = int(out[1].item())
+        return out[0][:n].cpu().numpy()
+
+    def rk_moe_fanout(self, p: torch.Tensor, tau: float, fence: bool = False, k_out=None, keep_out=None):
+        """Eq. (moe): p [n, 6] float32 Top-6 router weights -> (K_t [n] uint8, keep mask [n] uint8)."""
+        assert p.dtype == torch.float32 and p.dim() == 2 and p.shape[1] == 6 and p.is_contiguous()
+        n = p.shape[0]
+        if k_out is None:
+            k_out = torch.empty(n, dtype=torch.uint8, device=p.device)
+            keep_out = torch.empty(n, dtype=torch.uint8, device=p.device)
+        self.check(lib.rk_moe_fanout(self.handle, _ptr(p), n, float(tau), int(bool(fence)), _ptr(k_out), _ptr(keep_out),
+                                     _stream()))
+        return k_out, keep_out
 
     def rk_combine_offline(self, req, z_on_g, z_on_l, z_off, W_b, z=None, y=None):
         dev = z_on_g.device

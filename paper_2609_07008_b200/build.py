@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "librk.so")
-SOURCES = ["rk_host.cu", "rk_attn.cu", "rk_gemm.cu", "rk_stream.cu"]
+SOURCES = ["rk_host.cu", "rk_attn.cu", "rk_gemm.cu", "rk_stream.cu", "rk_policy.cu"]
 HEADERS = ["rk_ptx.cuh", "rk_internal.h", os.path.join("..", "..", "include", "rk.h")]
 
 

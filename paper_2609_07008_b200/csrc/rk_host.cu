@@ -839,6 +839,75 @@ rk_status rk_layer_stack_host(rk_ctx* ctx, int32_t n_layers, const rk_layer_io* 
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "stack synchronisation");
 }
 
+// ------------------------------------------------------------------------------------------
+// Selection rules: protected-row set (Eq. protected) and expert fan-out (Eq. moe)
+rk_status rk_protected_rows_workspace_bytes(int64_t n_rows, int32_t n_segs, size_t* out) {
+  if (!out) return RK_ERR_NULL;
+  if (n_rows <= 0 || n_rows >= ((int64_t)1 << 30) || n_segs <= 0) return RK_ERR_LAYOUT;
+  *out = policy_workspace_bytes(n_rows, n_segs);
+  return RK_OK;
+}
+
+rk_status rk_protected_rows(rk_ctx* ctx, const rk_layout* lay, const rk_policy* pol, const int32_t* dirty_rows,
+                            int64_t n_dirty, const float* scores, int32_t* rows_out, int64_t* count_out,
+                            void* workspace, size_t workspace_bytes, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!lay || !pol || !rows_out || !count_out || !workspace || (n_dirty > 0 && !dirty_rows))
+    return fail(ctx, RK_ERR_NULL, "null argument");
+  {
+    char msg[256] = {0};
+    rk_status s = rk_check_request(lay, nullptr, 0, msg, sizeof(msg));
+    // the layout-only part of the check: rows without artifact are what this call is about to protect
+    if (s != RK_OK && s != RK_ERR_ROWS) return fail(ctx, s, "%s", msg);
+  }
+  if (pol->edge_rows < 0 || pol->tail_rows < 0 || pol->budget_bp < 0 || pol->budget_bp > 10000)
+    return fail(ctx, RK_ERR_PROFILE, "policy out of range: edge_rows %d, tail_rows %lld, budget_bp %d", pol->edge_rows,
+                (long long)pol->tail_rows, pol->budget_bp);
+  if (n_dirty < 0) return fail(ctx, RK_ERR_ROWS, "n_dirty is negative");
+  const int S = lay->n_segs;
+  const int64_t T = lay->seg_off[S];
+  const size_t need = policy_workspace_bytes(T, S);
+  if (workspace_bytes < need) return fail(ctx, RK_ERR_WORKSPACE, "workspace too small: %zu < %zu", workspace_bytes, need);
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return fail(ctx, RK_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+  std::vector<int32_t> tab((size_t)(2 * S + 1));
+  int64_t req_end = 0;
+  for (int i = 0; i <= S; ++i) tab[(size_t)i] = (int32_t)lay->seg_off[i];
+  for (int i = 0; i < S; ++i) {
+    tab[(size_t)(S + 1 + i)] = (int32_t)lay->seg_delta[i];
+    req_end = std::max<int64_t>(req_end, lay->seg_delta[i] + lay->seg_off[i + 1] - lay->seg_off[i]);
+  }
+  PolicyHost h = {};
+  h.seg_tab_host = tab.data();
+  h.has_host = lay->seg_has_artifact;
+  h.n_segs = S;
+  h.T = T;
+  h.req_end = req_end;
+  h.tail_rows = pol->tail_rows;
+  h.edge_rows = pol->edge_rows;
+  h.budget_bp = pol->budget_bp;
+  h.dirty = dirty_rows;
+  h.n_dirty = n_dirty;
+  h.scores = scores;
+  h.rows_out = rows_out;
+  h.count_out = reinterpret_cast<long long*>(count_out);
+  h.workspace = workspace;
+  cudaError_t e = launch_protected_rows(h, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "protected-row kernels");
+  return RK_OK;
+}
+
+rk_status rk_moe_fanout(rk_ctx* ctx, const float* p, int64_t n, float tau, int32_t fence, uint8_t* k_out,
+                        uint8_t* keep_out, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (n < 0) return fail(ctx, RK_ERR_ROWS, "n is negative");
+  if (n > 0 && (!p || !k_out || !keep_out)) return fail(ctx, RK_ERR_NULL, "null argument");
+  if ((reinterpret_cast<uintptr_t>(p) & 7u) != 0) return fail(ctx, RK_ERR_LAYOUT, "router weights must be 8-byte aligned");
+  if (!(tau == tau)) return fail(ctx, RK_ERR_PROFILE, "tau is NaN");
+  cudaError_t e = launch_moe_fanout(p, n, tau, fence != 0, k_out, keep_out, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "fan-out kernel");
+  return RK_OK;
+}
+
 }  // extern "C"
 
 // ------------------------------------------------------------------------------------------

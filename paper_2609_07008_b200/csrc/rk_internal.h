@@ -86,4 +86,46 @@ cudaError_t launch_merge(int32_t n_parts, int64_t n_rh, const void* O_part, int3
 cudaError_t launch_combine(const void* z_on_g, const void* z_on_l, const void* z_off, const int32_t* inv_map,
                            int64_t T, int64_t width, void* z, int sm_count, cudaStream_t stream);
 
+// ---- selection rules (Eq. protected, Eq. moe) --------------------------------------------------
+constexpr uint8_t kPolicyStructural = 1, kPolicyCandidate = 2, kPolicyDirty = 4;
+
+struct PolicyState {
+  unsigned n_cand, n_struct_cand, blocks_done, n_top, k_rem, pad;
+  unsigned long long prefix;  // digits of the n_top-th largest (score,row) key found so far
+  unsigned hist[256];
+};
+
+struct PolicyParams {
+  const int32_t* seg_off;
+  const int32_t* seg_delta;
+  const uint8_t* seg_has_artifact;
+  const float* scores;
+  uint8_t* flags;
+  PolicyState* state;
+  unsigned* block_counts;
+  int32_t* rows_out;
+  long long* count_out;
+  long long req_end, tail_rows;
+  int32_t n_segs, T, edge_rows, budget_bp;
+};
+
+struct PolicyHost {
+  const int32_t* seg_tab_host;  // [seg_off (S+1) | seg_delta (S)]
+  const uint8_t* has_host;      // [S]
+  int32_t n_segs;
+  int64_t T, req_end, tail_rows;
+  int32_t edge_rows, budget_bp;
+  const int32_t* dirty;
+  int64_t n_dirty;
+  const float* scores;
+  int32_t* rows_out;
+  long long* count_out;
+  void* workspace;
+};
+
+size_t policy_workspace_bytes(int64_t T, int32_t n_segs);
+cudaError_t launch_protected_rows(const PolicyHost& h, cudaStream_t stream);
+cudaError_t launch_moe_fanout(const float* p, int64_t n, float tau, int fence, uint8_t* k_out, uint8_t* keep_out,
+                              cudaStream_t stream);
+
 }  // namespace rk

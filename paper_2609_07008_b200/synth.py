@@ -322,3 +322,39 @@ def sample_rows(layout: Layout, prot_rows: np.ndarray, n_random: int, seed: int,
     if n_random - n_half and len(unprot):
         picked += rng.choice(unprot, size=min(n_random - n_half, len(unprot)), replace=False).tolist()
     return np.unique(np.asarray(picked, dtype=np.int64))
+
+
+# ----------------------------------------------------------------------------------
+# inputs of the selection rules (Eq. protected, Eq. moe): seeded data only, no rule arithmetic
+# ----------------------------------------------------------------------------------
+
+def draw_policy_inputs(layout: Layout, seed: int, n_dirty: int = 64, tie_share: float = 0.05):
+    """Dirty rows (any order, with a few duplicates) and float32 Indexer scores with exact ties:
+    scores are standard normal, a `tie_share` of the rows is set to one of four fixed values."""
+    rng = np.random.default_rng(seed)
+    T = layout.n_rows
+    dirty = rng.integers(0, T, size=n_dirty).astype(np.int32)
+    if n_dirty >= 4:
+        dirty[-2:] = dirty[:2]
+    scores = rng.standard_normal(T).astype(np.float32)
+    n_tie = int(tie_share * T)
+    if n_tie:
+        idx = rng.choice(T, size=n_tie, replace=False)
+        scores[idx] = rng.choice(np.array([-0.5, 0.0, 0.25, 1.5], dtype=np.float32), size=n_tie)
+    return dirty, scores
+
+
+def draw_router_weights(n: int, seed: int, temperature: float = 1.5, tie_share: float = 0.02) -> np.ndarray:
+    """Top-6 router weights [n, 6] float32 in arbitrary slot order: six shares of a softmax over
+    random logits, scaled by the token's routed mass in (0.2, 0.9); a few rows carry exact ties."""
+    rng = np.random.default_rng(seed)
+    logits = rng.standard_normal((n, 6)) * temperature
+    e = np.exp(logits - logits.max(axis=1, keepdims=True))
+    p = e / e.sum(axis=1, keepdims=True) * rng.uniform(0.2, 0.9, size=(n, 1))
+    p = p.astype(np.float32)
+    n_tie = int(tie_share * n)
+    if n_tie:
+        rows = rng.choice(n, size=n_tie, replace=False)
+        a, b = rng.integers(0, 6, size=n_tie), rng.integers(0, 6, size=n_tie)
+        p[rows, a] = p[rows, b]
+    return p
