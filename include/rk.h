@@ -274,8 +274,9 @@ typedef struct rk_layer_buffers {
  * memory; pageable memory works but serialises), runs (2), (4), (5), copies y device->host and
  * synchronises `stream`.  Weights stay resident on the device.  Copies that the running kernel
  * does not need yet travel on an internal second stream beside it (the Local pass needs only kv
- * and q_l; q_g and the artifact arrive meanwhile; y returns in row chunks behind the shared
- * projection) and are ordered by device events, not by host polling (Section "Turning omitted
+ * and q_l; q_g and the artifact arrive meanwhile; the Global pass and everything after it run in
+ * two row ranges, and the y rows of the first range return while the second computes) and are
+ * ordered by device events, not by host polling (Section "Turning omitted
  * work into latency reduction": prefetch stream guarded by device events). */
 rk_status rk_layer_host(rk_ctx* ctx, const rk_request* req, const void* kv_host, const void* q_g_host,
                         const void* q_l_host, const void* z_off_host, const void* W_uv, const void* W_a,

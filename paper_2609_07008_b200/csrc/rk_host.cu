@@ -57,6 +57,16 @@ struct rk_request {
   float2* d_seg_cs = nullptr;
   AttnWorkItem* d_work_g = nullptr;
   AttnWorkItem* d_work_l = nullptr;
+  // rk_layer_host runs the Global pass in two row ranges [0, split_tok) and [split_tok, T) so that the
+  // first range's y travels to the host while the second computes; each range has its own tile list
+  int64_t split_tok = 0;  // 0: not split
+  AttnWorkItem* d_work_g_part[2] = {nullptr, nullptr};
+  int32_t n_tiles_g_part[2] = {0, 0};
+  // likewise the Local pass: a short first range of protected-row slots [0, split_slot) lets the pass
+  // start as soon as kv and that range's queries are on the device
+  int64_t split_slot = 0;
+  AttnWorkItem* d_work_l_part[2] = {nullptr, nullptr};
+  int32_t n_tiles_l_part[2] = {0, 0};
 };
 
 namespace {
@@ -106,12 +116,16 @@ rk_status make_tmap(const rk_ctx* ctx, CUtensorMap* m, const void* base, uint64_
   return RK_OK;
 }
 
+// tile_lo / tile_hi restrict the list to the row tiles [tile_lo, tile_hi) (-1: up to the last tile)
 void build_work(const std::vector<int32_t>& tok_pos, int hpt, const std::vector<int32_t>& seg_n,
-                const std::vector<int32_t>& seg_delta, int n_pairs, std::vector<AttnWorkItem>* out) {
+                const std::vector<int32_t>& seg_delta, int n_pairs, std::vector<AttnWorkItem>* out,
+                int64_t tile_lo = 0, int64_t tile_hi = -1) {
   const int64_t n_flat = (int64_t)tok_pos.size() * hpt;
-  const int64_t n_tiles = (n_flat + kAttnRowsPerPair - 1) / kAttnRowsPerPair;
+  const int64_t all_tiles = (n_flat + kAttnRowsPerPair - 1) / kAttnRowsPerPair;
+  if (tile_hi < 0 || tile_hi > all_tiles) tile_hi = all_tiles;
+  const int64_t n_tiles = tile_hi - tile_lo;
   std::vector<std::pair<int64_t, AttnWorkItem>> items((size_t)n_tiles);
-  for (int64_t t = 0; t < n_tiles; ++t) {
+  for (int64_t t = tile_lo; t < tile_hi; ++t) {
     const int64_t r0 = t * kAttnRowsPerPair, r1 = std::min<int64_t>(n_flat, r0 + kAttnRowsPerPair);
     const int64_t tok0 = r0 / hpt, tok1 = (r1 - 1) / hpt;
     int32_t maxpos = 0;
@@ -121,7 +135,7 @@ void build_work(const std::vector<int32_t>& tok_pos, int hpt, const std::vector<
       int64_t kmax = std::min<int64_t>(seg_n[i], (int64_t)maxpos - seg_delta[i] + 1);
       if (kmax > 0) cost += (kmax + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
     }
-    items[(size_t)t] = {cost, AttnWorkItem{(int32_t)t, maxpos}};
+    items[(size_t)(t - tile_lo)] = {cost, AttnWorkItem{(int32_t)t, maxpos}};
   }
   std::stable_sort(items.begin(), items.end(),
                    [](const auto& a, const auto& b) { return a.first > b.first; });
@@ -423,6 +437,38 @@ rk_status rk_request_create(rk_ctx* ctx, const rk_layout* lay, const int32_t* pr
   build_work(prot_pos, (int)ctx->local_heads.size(), seg_n, seg_delta32, ctx->n_pairs, &work_l);
   rq->n_tiles_g = (int32_t)work_g.size();
   rq->n_tiles_l = (int32_t)work_l.size();
+  std::vector<AttnWorkItem> work_part[2];
+  {  // two row ranges for rk_layer_host: the boundary must fall on a row-tile boundary of the Global pass
+    const int G = ctx->prof.n_groups;
+    int gcd = G, b = kAttnRowsPerPair;
+    while (b) { const int r = gcd % b; gcd = b; b = r; }
+    const int64_t unit = kAttnRowsPerPair / gcd;  // tokens per smallest whole number of tiles
+    const int64_t split = (T * 7 / 8) / unit * unit;
+    if (T >= 512 && split > 0 && split < T) {
+      rq->split_tok = split;
+      const int64_t tile_split = split * G / kAttnRowsPerPair;
+      build_work(row_pos, G, seg_n, seg_delta32, ctx->n_pairs, &work_part[0], 0, tile_split);
+      build_work(row_pos, G, seg_n, seg_delta32, ctx->n_pairs, &work_part[1], tile_split, -1);
+      rq->n_tiles_g_part[0] = (int32_t)work_part[0].size();
+      rq->n_tiles_g_part[1] = (int32_t)work_part[1].size();
+    }
+  }
+  std::vector<AttnWorkItem> work_lpart[2];
+  {
+    const int L = (int)ctx->local_heads.size();
+    int gcd = L, b = kAttnRowsPerPair;
+    while (b) { const int r = gcd % b; gcd = b; b = r; }
+    const int64_t unit = kAttnRowsPerPair / gcd;
+    const int64_t split = (n_prot / 8) / unit * unit;
+    if (n_prot >= 512 && split > 0 && split < n_prot) {
+      rq->split_slot = split;
+      const int64_t tile_split = split * L / kAttnRowsPerPair;
+      build_work(prot_pos, L, seg_n, seg_delta32, ctx->n_pairs, &work_lpart[0], 0, tile_split);
+      build_work(prot_pos, L, seg_n, seg_delta32, ctx->n_pairs, &work_lpart[1], tile_split, -1);
+      rq->n_tiles_l_part[0] = (int32_t)work_lpart[0].size();
+      rq->n_tiles_l_part[1] = (int32_t)work_lpart[1].size();
+    }
+  }
 
   cudaError_t e = upload(&rq->d_row_pos, row_pos);
   if (e == cudaSuccess) e = upload(&rq->d_prot_rows, prot);
@@ -432,6 +478,10 @@ rk_status rk_request_create(rk_ctx* ctx, const rk_layout* lay, const int32_t* pr
   if (e == cudaSuccess) e = upload(&rq->d_seg_cs, cs);
   if (e == cudaSuccess) e = upload(&rq->d_work_g, work_g);
   if (e == cudaSuccess) e = upload(&rq->d_work_l, work_l);
+  if (e == cudaSuccess && rq->split_tok > 0) e = upload(&rq->d_work_g_part[0], work_part[0]);
+  if (e == cudaSuccess && rq->split_tok > 0) e = upload(&rq->d_work_g_part[1], work_part[1]);
+  if (e == cudaSuccess && rq->split_slot > 0) e = upload(&rq->d_work_l_part[0], work_lpart[0]);
+  if (e == cudaSuccess && rq->split_slot > 0) e = upload(&rq->d_work_l_part[1], work_lpart[1]);
   if (e != cudaSuccess) {
     rk_request_destroy(rq);
     return cuda_fail(ctx, e, "request table upload");
@@ -450,6 +500,10 @@ rk_status rk_request_destroy(rk_request* rq) {
   cudaFree(rq->d_seg_cs);
   cudaFree(rq->d_work_g);
   cudaFree(rq->d_work_l);
+  cudaFree(rq->d_work_g_part[0]);
+  cudaFree(rq->d_work_g_part[1]);
+  cudaFree(rq->d_work_l_part[0]);
+  cudaFree(rq->d_work_l_part[1]);
   delete rq;
   return RK_OK;
 }
@@ -709,51 +763,90 @@ rk_status rk_layer_host(rk_ctx* ctx, const rk_request* rq, const void* kv_host, 
   const bool has_l = rq->A > 0;
   // The copy stream starts after everything already queued on `stream` (the staging buffers may
   // still be in use by an earlier call) and runs beside the kernels from then on: the Local pass
-  // needs only kv and q_l, so q_g and the artifact travel while it computes; y goes back in row
-  // chunks while the shared projection of the next chunk runs.  Ordering is by device events.
-  cudaError_t e = cudaEventRecord(ctx->ev[0], st);
+  // needs only kv and q_l, so q_g and the artifact travel while it computes; the rest of the layer
+  // runs in two row ranges, and the y rows of the first go back while the second computes.
+  // Ordering is by device events.
+  // first on the wire: kv and the queries of the first Local range, alone, so that the Local pass can
+  // start; the copy stream follows with the rest of q_l, then q_g, then the artifact
+  const size_t ql_row = (size_t)L * kDQK * 2;
+  const int64_t slot0 = (has_l && rq->split_slot > 0) ? rq->split_slot : rq->A;  // protected-row slots sent up front
+  cudaError_t e = cudaMemcpyAsync(dev->kv, kv_host, (size_t)T * kDQK * 2, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && has_l) e = cudaMemcpyAsync(dev->q_l, q_l_host, (size_t)slot0 * ql_row, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaEventRecord(ctx->ev[0], st);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(cp, ctx->ev[0], 0);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(dev->kv, kv_host, (size_t)T * kDQK * 2, cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess && has_l)
-    e = cudaMemcpyAsync(dev->q_l, q_l_host, (size_t)rq->A * L * kDQK * 2, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && slot0 < rq->A)
+    e = cudaMemcpyAsync(reinterpret_cast<uint8_t*>(dev->q_l) + (size_t)slot0 * ql_row,
+                        reinterpret_cast<const uint8_t*>(q_l_host) + (size_t)slot0 * ql_row, (size_t)(rq->A - slot0) * ql_row,
+                        cudaMemcpyHostToDevice, cp);
+  if (e == cudaSuccess) e = cudaEventRecord(ctx->ev[6], cp);
   if (e == cudaSuccess) e = cudaMemcpyAsync(dev->q_g, q_g_host, (size_t)T * G * kDQK * 2, cudaMemcpyHostToDevice, cp);
   if (e == cudaSuccess) e = cudaEventRecord(ctx->ev[1], cp);
   if (e == cudaSuccess && rq->n_off_rows > 0 && z_off_host)
     e = cudaMemcpyAsync(dev->z_off, z_off_host, (size_t)rq->n_off_rows * width * 2, cudaMemcpyHostToDevice, cp);
   if (e == cudaSuccess) e = cudaEventRecord(ctx->ev[2], cp);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "host to device copy");
+  if (!aligned16(dev->kv) || !aligned16(dev->q_g) || !aligned16(dev->O_g) || !aligned16(dev->z_on_g) || !aligned16(dev->z) ||
+      !aligned16(dev->y) || (reinterpret_cast<uintptr_t>(dev->workspace) & 255u))
+    return fail(ctx, RK_ERR_ALIGN, "device buffers must be 16-byte aligned and the workspace 256-byte aligned");
+  if (dev->workspace_bytes < proj_ws_bytes(rq)) return fail(ctx, RK_ERR_WORKSPACE, "workspace too small: need %zu bytes", proj_ws_bytes(rq));
+  const int H = ctx->prof.n_heads, ro = ctx->prof.o_rank;
   rk_status s = RK_OK;
-  if (has_l) s = rk_mla_online_attn(ctx, rq, dev->kv, nullptr, dev->q_l, nullptr, nullptr, dev->O_l, dev->lse_l, stream);
-  if (s != RK_OK) return s;
+  if (has_l) {  // Local pass and the Local half of the first projection: need kv, q_l only
+    if (!aligned16(dev->q_l) || !aligned16(dev->O_l)) return fail(ctx, RK_ERR_ALIGN, "device buffers must be 16-byte aligned");
+    if (slot0 < rq->A) {
+      s = attn_pass(ctx, rq, dev->kv, dev->q_l, rq->A, L, rq->d_prot_rows, rq->d_work_l_part[0], rq->n_tiles_l_part[0],
+                    dev->O_l, dev->lse_l, st);
+      e = cudaStreamWaitEvent(st, ctx->ev[6], 0);
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
+      if (s == RK_OK)
+        s = attn_pass(ctx, rq, dev->kv, dev->q_l, rq->A, L, rq->d_prot_rows, rq->d_work_l_part[1], rq->n_tiles_l_part[1],
+                      dev->O_l, dev->lse_l, st);
+    } else {
+      s = attn_pass(ctx, rq, dev->kv, dev->q_l, rq->A, L, rq->d_prot_rows, rq->d_work_l, rq->n_tiles_l, dev->O_l,
+                    dev->lse_l, st);
+    }
+    if (s == RK_OK)
+      s = rk_group_sliced_proj(ctx, rq, nullptr, dev->O_l, W_uv, W_a, nullptr, dev->z_on_l, dev->workspace,
+                               dev->workspace_bytes, stream);
+    if (s != RK_OK) return s;
+  }
   e = cudaStreamWaitEvent(st, ctx->ev[1], 0);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
-  s = rk_mla_online_attn(ctx, rq, dev->kv, dev->q_g, nullptr, dev->O_g, dev->lse_g, nullptr, nullptr, stream);
-  if (s == RK_OK)
-    s = rk_group_sliced_proj(ctx, rq, dev->O_g, has_l ? dev->O_l : nullptr, W_uv, W_a, dev->z_on_g,
-                             has_l ? dev->z_on_l : nullptr, dev->workspace, dev->workspace_bytes, stream);
-  if (s != RK_OK) return s;
-  e = cudaStreamWaitEvent(st, ctx->ev[2], 0);
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
-  // restore-and-replace + W_b in up to four row chunks; each chunk's y is copied out behind it
-  const int n_chunks = T >= 4 * 1024 ? 4 : 1;
-  const int64_t rows_per = ((T + n_chunks - 1) / n_chunks + 127) / 128 * 128;
-  const uint8_t* zg = reinterpret_cast<const uint8_t*>(dev->z_on_g);
+  // Global pass, Global half of the first projection, restore-and-replace and W_b per row range; the y
+  // rows of a range are copied out while the next range computes
+  const int n_chunks = rq->split_tok > 0 ? 2 : 1;
+  const uint8_t* Og = reinterpret_cast<const uint8_t*>(dev->O_g);
+  uint8_t* og = reinterpret_cast<uint8_t*>(dev->workspace);  // per-head W_uv output of the Global heads
+  uint8_t* zg = reinterpret_cast<uint8_t*>(dev->z_on_g);
   const uint8_t* zo = reinterpret_cast<const uint8_t*>(dev->z_off);
   uint8_t* zz = reinterpret_cast<uint8_t*>(dev->z);
   uint8_t* yy = reinterpret_cast<uint8_t*>(dev->y);
   for (int c = 0; c < n_chunks; ++c) {
-    const int64_t r0 = c * rows_per, r1 = std::min<int64_t>(T, r0 + rows_per);
-    if (r0 >= r1) break;
-    e = launch_combine(zg + r0 * width * 2, dev->z_on_l, zo ? zo + r0 * width * 2 : nullptr, rq->d_inv_map + r0, r1 - r0,
-                       (int64_t)width, zz + r0 * width * 2, ctx->sm_count, st);
+    const int64_t r0 = c == 0 ? 0 : rq->split_tok, r1 = (n_chunks == 2 && c == 0) ? rq->split_tok : T;
+    const int64_t n = r1 - r0;
+    s = attn_pass(ctx, rq, dev->kv, dev->q_g, T, G, nullptr, n_chunks == 2 ? rq->d_work_g_part[c] : rq->d_work_g,
+                  n_chunks == 2 ? rq->n_tiles_g_part[c] : rq->n_tiles_g, dev->O_g, dev->lse_g, st);
+    if (s == RK_OK)
+      s = run_gemm(ctx, Og + (size_t)r0 * G * kDLatent * 2, n, (int64_t)G * kDLatent, W_uv, (int64_t)H * kDV, kDLatent,
+                   og + (size_t)r0 * G * kDV * 2, (int64_t)G * kDV, (int)n, kDV, kDLatent, ctx->off_uv_g, G, st);
+    if (s == RK_OK)
+      s = run_gemm(ctx, og + (size_t)r0 * G * kDV * 2, n, (int64_t)G * kDV, W_a, (int64_t)G * ro, kGroup * kDV,
+                   zg + (size_t)r0 * width * 2, (int64_t)G * ro, (int)n, ro, kDV, ctx->off_wa_g, G, st);
+    if (s != RK_OK) return s;
+    if (c == 0) {  // the artifact has to be there from here on
+      e = cudaStreamWaitEvent(st, ctx->ev[2], 0);
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
+    }
+    e = launch_combine(zg + (size_t)r0 * width * 2, dev->z_on_l, zo ? zo + (size_t)r0 * width * 2 : nullptr, rq->d_inv_map + r0, n,
+                       (int64_t)width, zz + (size_t)r0 * width * 2, ctx->sm_count, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "combine launch");
-    s = run_gemm(ctx, zz + r0 * width * 2, r1 - r0, (int64_t)width, W_b, dm, (int64_t)width, yy + r0 * dm * 2, dm,
-                 (int)(r1 - r0), (int)dm, (int)width, ctx->off_wb, 1, st);
+    s = run_gemm(ctx, zz + (size_t)r0 * width * 2, n, (int64_t)width, W_b, dm, (int64_t)width, yy + (size_t)r0 * dm * 2, dm, (int)n,
+                 (int)dm, (int)width, ctx->off_wb, 1, st);
     if (s != RK_OK) return s;
     e = cudaEventRecord(ctx->ev[3 + c], st);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(cp, ctx->ev[3 + c], 0);
     if (e == cudaSuccess)
-      e = cudaMemcpyAsync(reinterpret_cast<uint8_t*>(y_host) + r0 * dm * 2, yy + r0 * dm * 2, (size_t)(r1 - r0) * dm * 2,
+      e = cudaMemcpyAsync(reinterpret_cast<uint8_t*>(y_host) + (size_t)r0 * dm * 2, yy + (size_t)r0 * dm * 2, (size_t)n * dm * 2,
                           cudaMemcpyDeviceToHost, cp);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "device to host copy");
   }

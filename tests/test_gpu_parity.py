@@ -229,6 +229,30 @@ def test_end_to_end_tiny_honest_artifact(rk, regime):
     assert torch.equal(y_h, y.cpu())
 
 
+def test_layer_host_row_ranges_equal_device_path(rk):
+    """rk_layer_host runs the Local pass and everything from the Global pass on in two row ranges each
+    (so that copies overlap kernels); the result is bit-identical to the call-by-call device path."""
+    w = synth.make_custom([1500, 900, 700], 200, n_heads=16, n_groups=2, o_rank=256, d_model=512, pct_bp=3000, seed=9)
+    ctx, req = make(rk, w)
+    assert req.A >= 512 and w.layout.n_rows >= 512          # both passes are split at these sizes
+    to_device(w)
+    O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
+    z_on_g, z_on_l = ctx.rk_group_sliced_proj(req, O_g, O_l, w.w_uv, w.w_a)
+    z, y = ctx.rk_combine_offline(req, z_on_g, z_on_l, w.z_off, w.w_b)
+    ctx.rk_poll_status()
+    bufs = ctx.alloc_layer_buffers(req, "cuda")
+    pin = lambda t: t.cpu().pin_memory()
+    y_h = torch.empty((w.layout.n_rows, w.profile.d_model), dtype=torch.bfloat16).pin_memory()
+    for _ in range(2):                                       # a second call reuses the staging buffers
+        y_h.zero_()
+        ctx.rk_layer_host(req, pin(w.kv), pin(w.q_g), pin(w.q_l), pin(w.z_off), w.w_uv, w.w_a, w.w_b, bufs, y_h)
+        ctx.rk_poll_status()
+        assert torch.equal(y_h, y.cpu())
+    rows = synth.sample_rows(w.layout, w.prot_rows, 16, seed=1)
+    exp = oracle_online(w, rows)
+    assert_close(f64(y_h[rows]), exp["y"], "y (host path, sampled rows)")
+
+
 # -- edge cases -------------------------------------------------------------------------------------------
 
 def _layer(rk, w):
