@@ -32,9 +32,18 @@
 namespace rk {
 #ifdef RK_TRACE
 __device__ long long g_trace[4 * 16384];
-#define RK_TR(role, tag) do { if (blockIdx.x == 0 && lane == 0 && tr_n[role] < 8190) { g_trace[(role) * 16384 + 2 * tr_n[role]] = (tag); g_trace[(role) * 16384 + 2 * tr_n[role] + 1] = clock64(); ++tr_n[role]; } } while (0)
+// records (tag, clock64) pairs of CTA 0; the events of the first ((debug >> 8) << 6) key tiles are skipped
+// so that a window late in a long launch can be looked at
+#define RK_TR(role, tag) do { if (blockIdx.x == 0 && lane == 0) { if (tr_skip[role] > 0) --tr_skip[role]; else if (tr_n[role] < 8190) { g_trace[(role) * 16384 + 2 * tr_n[role]] = (tag); g_trace[(role) * 16384 + 2 * tr_n[role] + 1] = clock64(); ++tr_n[role]; } } } while (0)
+// cheap wait-time accumulators (clock deltas summed in registers, written once at the end of CTA 0)
+#define RK_ACC_T0() const long long acc_t0 = clock64()
+#define RK_ACC(i) do { acc[i] += clock64() - acc_t0; } while (0)
+#define RK_ACC_DUMP(role, n) do { if (blockIdx.x == 0 && lane == 0) for (int i_ = 0; i_ < (n); ++i_) g_trace[3 * 16384 + 32 * (role) + i_] = acc[i_]; } while (0)
 #else
 #define RK_TR(role, tag) do { } while (0)
+#define RK_ACC_T0() do { } while (0)
+#define RK_ACC(i) do { } while (0)
+#define RK_ACC_DUMP(role, n) do { } while (0)
 #endif
 namespace {
 
@@ -196,6 +205,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
   const uint64_t limit = p.wait_ns;
 #ifdef RK_TRACE
   int tr_n[4] = {0, 0, 0, 0};
+  const int tr_tiles = (p.debug >> 8) << 6;  // events per key tile: issuer 23, softmax 5, producer 9
+  int tr_skip[4] = {23 * tr_tiles, 5 * tr_tiles, 9 * tr_tiles, 0};
+  if (p.debug & 16) tr_skip[0] = tr_skip[1] = tr_skip[2] = 0x7fffffff;  // accumulators only, no event records
+  long long acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+  const long long acc_start = clock64();
 #endif
 
   for (int i = threadIdx.x; i < 512; i += kAttnThreads) reinterpret_cast<volatile unsigned long long*>(smem + kOffXchg)[i] = 0ull;
@@ -247,9 +261,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     auto fill = [&](int col0, int col1, int row, int w) -> bool {
       const uint32_t s = rp.stage();
       if (rp.it >= (uint32_t)kStages) {
+        RK_ACC_T0();
         if (!mbar_wait_bounded<false>(bar(kBarRingEmpty + s), rp.parity() ^ 1u, limit, abort_flag, p.status,
                                       W_RINGEMPTY, w))
           return false;
+        RK_ACC(0);
       }
       if (p.debug & 8) {  // test switch: leave the stage empty so that the consumer's bounded wait expires
         rp.advance();
@@ -333,6 +349,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       }
       if (ok && prev_row0 >= 0) ok = load_v(prev_row0, prev_kb, w);
     }
+#ifdef RK_TRACE
+    acc[1] = clock64() - acc_start;
+    RK_ACC_DUMP(2, 2);
+#endif
     // drain: every stage this CTA filled must have been released by the tensor core, and the
     // last Q tile must be free, before the CTA may exit
     if (ok && n_done > 0)
@@ -377,23 +397,32 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         auto issue_qk = [&](bool first_of_seg, bool last_of_seg, uint32_t rb) -> bool {
           RK_TR(0, 1);
           if (first_of_seg) {
+            RK_ACC_T0();
             if (!mbar_wait_bounded<true>(bar(kBarQrReady + rb), (qr_ready_phases >> rb) & 1u, limit, abort_flag,
                                          p.status, W_QRREADY, w))
               return false;
             qr_ready_phases ^= (1u << rb);
+            RK_ACC(0);
           }
           if (s_writes > 0) {  // one score buffer: the softmax warps must have read the previous key tile's scores
+            RK_ACC_T0();
             if (!mbar_wait_bounded<true>(bar(kBarSFree), (s_writes - 1) & 1u, limit, abort_flag, p.status, W_SFREE, w))
               return false;
             tc_fence_after_sync();
+            RK_ACC(1);
           }
           ++s_writes;
           const uint32_t tmem_s = tmem_base + kColS;
 #pragma unroll 1
           for (int st = 0; st < 5; ++st) {
             const uint32_t s = rp.stage();
-            if (!mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
-              return false;
+            RK_TR(0, 30 + st);
+            {
+              RK_ACC_T0();
+              if (!mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
+                return false;
+              RK_ACC(2 + st);
+            }
             const uint32_t b_addr = smem_base + kOffRing + s * kStageBytes;
             RK_TR(0, 10 + st);
             if (elect_one()) {
@@ -437,8 +466,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           return true;
         };
         auto issue_pv = [&]() -> bool {
-          if (!mbar_wait_bounded<true>(bar(kBarPReady), p_ready_phase, limit, abort_flag, p.status, W_PREADY, w))
-            return false;
+          {
+            RK_ACC_T0();
+            if (!mbar_wait_bounded<true>(bar(kBarPReady), p_ready_phase, limit, abort_flag, p.status, W_PREADY, w))
+              return false;
+            RK_ACC(7);
+          }
           p_ready_phase ^= 1;
           tc_fence_after_sync();
           RK_TR(0, 3);
@@ -446,8 +479,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           for (int q = 0; q < 4; ++q) {
             const int kh = q >> 1, h = q & 1;
             const uint32_t s = rp.stage();
-            if (!mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
-              return false;
+            RK_TR(0, 40 + q);
+            {
+              RK_ACC_T0();
+              if (!mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
+                return false;
+              RK_ACC(8 + q);
+            }
             const uint32_t b_addr = smem_base + kOffRing + s * kStageBytes;
             const uint32_t tmem_o = tmem_base + kColO + (uint32_t)h * 128u;
             RK_TR(0, 20 + q);
@@ -466,6 +504,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             rp.advance();
           }
           ++kt_pv;
+#ifdef RK_TRACE
+          acc[13] += 1;
+#endif
           RK_TR(0, 4);
           return true;
         };
@@ -483,6 +524,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         }
         while (ok && kt_pv < kt_issued) ok = issue_pv();
       }
+#ifdef RK_TRACE
+      acc[12] = clock64() - acc_start;
+      RK_ACC_DUMP(0, 16);
+#endif
     }
   } else if (warp == 2) {
     // ------------------------------ query relocation ----------------------------------------
@@ -612,7 +657,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         for (int kb = 0; kb < it.kmax && ok; kb += kAttnKeysPerTile, ++kt) {
           int nv = lim - (kb + part * 64) + 1;
           nv = nv < 0 ? 0 : (nv > 64 ? 64 : nv);
-          ok = mbar_wait_bounded<false>(bar(kBarSFull), s_full_phase, limit, abort_flag, p.status, W_SFULL, w);
+          {
+            RK_ACC_T0();
+            ok = mbar_wait_bounded<false>(bar(kBarSFull), s_full_phase, limit, abort_flag, p.status, W_SFULL, w);
+            RK_ACC(0);
+          }
           s_full_phase ^= 1;
           if (!ok) break;
           tc_fence_after_sync();
@@ -649,7 +698,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           }
           const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
           float mxo = mx;
-          if (!(p.debug & 4)) ok = quad_exchange_max(xbuf, part, m, ++xseq, mx, mxo, limit, abort_flag, p.status, w);
+          {
+            RK_ACC_T0();
+            if (!(p.debug & 4)) ok = quad_exchange_max(xbuf, part, m, ++xseq, mx, mxo, limit, abort_flag, p.status, w);
+            RK_ACC(1);
+          }
           if (!ok) break;
           if (warp == 4) RK_TR(1, 2);
           const float mt = mxo * scale;
@@ -686,7 +739,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           if (warp == 4) RK_TR(1, 3);
           // P buffer and O are free once the previous PV has completed
           if (kt > 0) {
-            ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
+            {
+              RK_ACC_T0();
+              ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
+              RK_ACC(2);
+            }
             pv_done_phase ^= 1;
             if (!ok) break;
             tc_fence_after_sync();
@@ -753,6 +810,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         p.lse[r] = (l_tot > 0.f) ? (m_run + log2f(l_tot)) * 0.69314718055994530942f : -INFINITY;
       tc_fence_before_sync();
     }
+#ifdef RK_TRACE
+    acc[3] = clock64() - acc_start;
+    if (warp == 4) RK_ACC_DUMP(1, 4);
+#endif
   }
 
   // ------------------------------ teardown ---------------------------------------------------

@@ -358,3 +358,35 @@ def draw_router_weights(n: int, seed: int, temperature: float = 1.5, tie_share: 
         a, b = rng.integers(0, 6, size=n_tie), rng.integers(0, 6, size=n_tie)
         p[rows, a] = p[rows, b]
     return p
+
+
+def make_random_request(seed: int, n_heads: int = 16, n_groups: int = 2, o_rank: int = 256, d_model: int = 512,
+                        regime: str = "sharp", device="cpu") -> Workload:
+    """A seeded irregular request for edge-case parity: 2-7 segments whose lengths mix tile-boundary
+    values (1, 2, 63..65, 127..129, 255..257) with random ones, a random request order with random gaps
+    between segments, some segments in the middle without artifact (new rows), a short query suffix
+    last in the request, and a random share of protected document rows."""
+    rng = np.random.default_rng(np.random.PCG64(1000 + seed))
+    special = [1, 2, 63, 64, 65, 127, 128, 129, 255, 256, 257]
+    n_docs = int(rng.integers(2, 7))
+    lens = [int(rng.choice(special)) if rng.random() < 0.6 else int(rng.integers(3, 600)) for _ in range(n_docs)]
+    lens.append(int(rng.integers(1, 80)))                    # query suffix, packed last
+    has = np.ones(n_docs + 1, dtype=np.uint8)
+    has[n_docs] = 0
+    for i in range(n_docs):
+        if rng.random() < 0.2:
+            has[i] = 0                                       # a new (uncached) segment in the middle
+    if has[:n_docs].sum() == 0:
+        has[0] = 1
+    order = list(rng.permutation(n_docs)) + [n_docs]         # request order; the query comes last
+    delta = np.zeros(n_docs + 1, dtype=np.int64)
+    run = int(rng.integers(0, 3)) * int(rng.integers(0, 40))
+    for i in order:
+        delta[i] = run
+        run += lens[i] + (int(rng.integers(0, 50)) if rng.random() < 0.4 else 0)
+    seg_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    layout = Layout(seg_off=seg_off, seg_delta=delta, seg_has_artifact=has)
+    prot = draw_protected_rows(layout, int(rng.integers(0, 3000)), rng)
+    profile = Profile(n_heads=n_heads, n_groups=n_groups, o_rank=o_rank, d_model=d_model,
+                      global_heads=draw_global_heads(n_groups, rng), sm_scale=float(1.0 / np.sqrt(D_V + D_ROPE)))
+    return make_tensors("random", profile, layout, prot, seed, device=device, regime=regime)

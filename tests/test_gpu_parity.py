@@ -253,6 +253,34 @@ def test_layer_host_row_ranges_equal_device_path(rk):
     assert_close(f64(y_h[rows]), exp["y"], "y (host path, sampled rows)")
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_irregular_requests_every_row(rk, seed):
+    """Seeded irregular requests (segment lengths on and around tile boundaries, length-1 segments, gaps,
+    shuffled request order, uncached segments in the middle): every row of every stage against the checker."""
+    w = synth.make_random_request(seed)
+    lay = w.layout
+    rows = np.arange(lay.n_rows)
+    exp = oracle_online(w, rows)
+    ctx, req = make(rk, w)
+    to_device(w)
+    O_g, lse_g, O_l, lse_l = ctx.rk_mla_online_attn(req, w.kv, w.q_g, w.q_l)
+    z_on_g, z_on_l = ctx.rk_group_sliced_proj(req, O_g, O_l, w.w_uv, w.w_a)
+    z, y = ctx.rk_combine_offline(req, z_on_g, z_on_l, w.z_off, w.w_b)
+    ctx.rk_poll_status()
+    assert_close(f64(O_g), exp["O_g"], "O_g")
+    assert np.abs(f64(lse_g) - exp["lse_g"]).max() <= 5e-3
+    assert_close(f64(O_l), exp["O_l"], "O_l")
+    assert_close(f64(z), exp["z"], "z")
+    assert_close(f64(y), exp["y"], "y")
+    # the same request through the host-buffer entry point gives the same bits
+    bufs = ctx.alloc_layer_buffers(req, "cuda")
+    pin = lambda t: t.cpu().pin_memory()
+    y_h = torch.empty((lay.n_rows, w.profile.d_model), dtype=torch.bfloat16).pin_memory()
+    ctx.rk_layer_host(req, pin(w.kv), pin(w.q_g), pin(w.q_l), pin(w.z_off), w.w_uv, w.w_a, w.w_b, bufs, y_h)
+    ctx.rk_poll_status()
+    assert torch.equal(y_h, y.cpu())
+
+
 # -- edge cases -------------------------------------------------------------------------------------------
 
 def _layer(rk, w):
