@@ -25,7 +25,9 @@ struct GemmSmem {
   static constexpr uint32_t kABytes = kBM * kBK * 2;  // 16 KB
   static constexpr uint32_t kBBytes = BN * kBK * 2;
   static constexpr uint32_t kStageBytes = kABytes + kBBytes;
-  static constexpr uint32_t kOffBars = kStages * kStageBytes;
+  static constexpr uint32_t kOffCStage = kStages * kStageBytes;  // two [128 rows x 128 B] output staging tiles
+  static constexpr uint32_t kCStageBytes = kBM * 128;
+  static constexpr uint32_t kOffBars = kOffCStage + 2 * kCStageBytes;
   // full[kStages], empty[kStages], acc_full[2], acc_empty[2]
   static constexpr uint32_t kOffTmemPtr = kOffBars + (2 * kStages + 4) * 8;
   static constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
@@ -34,8 +36,10 @@ struct GemmSmem {
 
 enum { WG_FULL = 31, WG_EMPTY, WG_ACC_FULL, WG_ACC_EMPTY };
 
-// Persistent: each CTA walks output tiles t = blockIdx.x, + gridDim.x, ... (column tile fastest, so
-// CTAs running at the same time share A row blocks and the whole of B through L2).  Two TMEM
+// Persistent: each CTA walks output tiles t = blockIdx.x, + gridDim.x, ... ordered row block, batch, column
+// tile (fastest), so the CTAs running at the same time cover a few 128-row blocks over the full output
+// width: they share those A rows and the whole of B through L2, and their stores fill whole output rows
+// at about the same time instead of 512-byte pieces scattered over every row of the tensor.  Two TMEM
 // accumulator buffers let the epilogue of tile i overlap the main loop of tile i + 1.
 template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1) rk_gemm_kernel(const __grid_constant__ GemmParams p) {
@@ -55,8 +59,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) rk_gemm_kernel(const __grid_c
 
   const int n_tiles_n = (p.N + BN - 1) / BN;
   const int n_tiles_m = (p.M + kBM - 1) / kBM;
-  const int tiles_per_batch = n_tiles_n * n_tiles_m;
-  const int n_tiles = tiles_per_batch * p.n_batches;
+  const int tiles_per_row_block = n_tiles_n * p.n_batches;  // all batches and column tiles of one 128-row block
+  const int n_tiles = tiles_per_row_block * n_tiles_m;
   const int k_chunks = p.K / kBK;
   constexpr uint32_t kTmemCols = 2 * BN;  // 256 or 512: power of two
 
@@ -91,9 +95,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) rk_gemm_kernel(const __grid_c
     uint32_t it = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-      const int batch = t / tiles_per_batch;
-      const int rem = t - batch * tiles_per_batch;
-      const int m0 = (rem / n_tiles_n) * kBM, n0 = (rem % n_tiles_n) * BN;
+      const int mb = t / tiles_per_row_block;
+      const int rem = t - mb * tiles_per_row_block;
+      const int batch = rem / n_tiles_n;
+      const int m0 = mb * kBM, n0 = (rem % n_tiles_n) * BN;
       const GemmBatch bt = p.batches[batch];
       for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
         const uint32_t s = it % kStages;
@@ -150,45 +155,61 @@ __global__ void __launch_bounds__(kGemmThreads, 1) rk_gemm_kernel(const __grid_c
       }
     }
   } else if (warp >= 4) {
-    // ---- epilogue: TMEM -> registers -> bf16 -> global, one row per thread ----
+    // ---- epilogue: TMEM -> registers -> bf16 -> swizzled shared-memory tile -> TMA store ----
+    // One row per thread.  64 output columns at a time go through one of two 16 KB staging tiles, so the
+    // stores reach memory as whole 128-byte lines of 128 rows (a thread's own 16-byte stores to rows a
+    // whole matrix row apart held the short-K projections at 40 % of the memory rate).
     const int L = threadIdx.x - 128;
     const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
-    uint32_t tile_i = 0;
+    uint32_t tile_i = 0, chunk_i = 0;
     bool ok = true;
+    if (L == 0) tma_prefetch_desc(&p.tm_c);
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
       const uint32_t b = tile_i & 1u;
-      const int batch = t / tiles_per_batch;
-      const int rem = t - batch * tiles_per_batch;
-      const int m0 = (rem / n_tiles_n) * kBM, n0 = (rem % n_tiles_n) * BN;
+      const int mb = t / tiles_per_row_block;
+      const int rem = t - mb * tiles_per_row_block;
+      const int batch = rem / n_tiles_n;
+      const int m0 = mb * kBM, n0 = (rem % n_tiles_n) * BN;
       const GemmBatch bt = p.batches[batch];
       ok = mbar_wait_bounded<false>(acc_full_bar(b), (tile_i >> 1) & 1u, limit, abort_flag, p.status, WG_ACC_FULL, t);
+      // the four warps leave together or not at all: the barriers below have no time limit of their own
+      ok = named_barrier_and(1, 128, ok);
       if (!ok) break;
       tc_fence_after_sync();
-      const int row = m0 + L;
-      __nv_bfloat16* crow =
-          reinterpret_cast<__nv_bfloat16*>(p.C) + (size_t)(row < p.M ? row : 0) * p.ldc + bt.c_col0 + n0;
 #pragma unroll 1
-      for (int cc = 0; cc < BN; cc += 32) {
-        uint32_t o[32];
+      for (int cc = 0; cc < BN; cc += 64, ++chunk_i) {
+        uint32_t o[64];
         tmem_ld_x32(tmem_base + lane_base + b * BN + cc, o);
+        tmem_ld_x32(tmem_base + lane_base + b * BN + cc + 32, o + 32);
         tmem_wait_ld();
-        if (row < p.M && n0 + cc < p.N) {
-          uint4* dst = reinterpret_cast<uint4*>(crow + cc);
+        if (cc + 64 >= BN) {  // the accumulator is in registers: hand it back to the tensor core
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty_bar(b));
+        }
+        const uint32_t buf = chunk_i & 1u;
+        // the store that last read this staging tile (two chunks ago) must have finished reading it
+        if (L == 0) bulk_wait_group_read<1>();
+        named_barrier_sync(1, 128);
+        uint8_t* stage = smem + S::kOffCStage + buf * S::kCStageBytes;
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            uint4 v;
-            v.x = pack_bf16(__uint_as_float(o[8 * e + 0]), __uint_as_float(o[8 * e + 1]));
-            v.y = pack_bf16(__uint_as_float(o[8 * e + 2]), __uint_as_float(o[8 * e + 3]));
-            v.z = pack_bf16(__uint_as_float(o[8 * e + 4]), __uint_as_float(o[8 * e + 5]));
-            v.w = pack_bf16(__uint_as_float(o[8 * e + 6]), __uint_as_float(o[8 * e + 7]));
-            dst[e] = v;
-          }
+        for (int e = 0; e < 8; ++e) {
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(o[8 * e + 0]), __uint_as_float(o[8 * e + 1]));
+          v.y = pack_bf16(__uint_as_float(o[8 * e + 2]), __uint_as_float(o[8 * e + 3]));
+          v.z = pack_bf16(__uint_as_float(o[8 * e + 4]), __uint_as_float(o[8 * e + 5]));
+          v.w = pack_bf16(__uint_as_float(o[8 * e + 6]), __uint_as_float(o[8 * e + 7]));
+          *reinterpret_cast<uint4*>(stage + sw128_offset((uint32_t)L, (uint32_t)e)) = v;
+        }
+        fence_proxy_async_smem();
+        named_barrier_sync(1, 128);
+        if (L == 0 && n0 + cc < p.N) {
+          tma_store_2d(&p.tm_c, smem_base + S::kOffCStage + buf * S::kCStageBytes, bt.c_col0 + n0 + cc, m0);
+          bulk_commit_group();
         }
       }
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty_bar(b));
     }
+    if (L == 0) bulk_wait_group<0>();  // the staging tiles must outlive the last stores
   }
   __syncwarp();
   tc_fence_before_sync();

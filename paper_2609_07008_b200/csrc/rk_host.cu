@@ -678,6 +678,8 @@ static rk_status run_gemm(rk_ctx* ctx, const void* A, int64_t a_rows, int64_t a_
   if (s != RK_OK) return s;
   s = make_tmap(ctx, &p.tm_b, B, (uint64_t)b_rows, (uint64_t)b_cols, (uint64_t)b_cols, 64, (uint32_t)bn);
   if (s != RK_OK) return s;
+  s = make_tmap(ctx, &p.tm_c, C, (uint64_t)M, (uint64_t)ldc, (uint64_t)ldc, 64, 128);
+  if (s != RK_OK) return s;
   p.C = C;
   p.batches = ctx->d_batches + batch_off;
   p.status = ctx->d_status;

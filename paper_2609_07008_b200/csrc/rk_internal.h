@@ -65,6 +65,7 @@ struct GemmBatch {
 struct GemmParams {
   CUtensorMap tm_a;  // [M rows][a_cols] box 64 x 128
   CUtensorMap tm_b;  // [b_rows][b_cols] box 64 x BN
+  CUtensorMap tm_c;  // [M rows][ldc] box 64 x 128 (epilogue stores)
   void* C;
   const GemmBatch* batches;
   DeviceStatus* status;
