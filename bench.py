@@ -467,7 +467,8 @@ def main():
         comb_bytes = 3 * req.T * width * 2
         breakdown = dict(sliced_proj_ms=t_proj, sliced_proj_tflops=fl_proj / t_proj / 1e9,
                          combine_ms=t_comb, combine_gbs=comb_bytes / t_comb / 1e6,
-                         wb_gemm_ms=t_cwb - t_comb, wb_gemm_tflops=fl_wb / (t_cwb - t_comb) / 1e9)
+                         wb_gemm_ms=t_cwb - t_comb, wb_gemm_tflops=fl_wb / (t_cwb - t_comb) / 1e9,
+                         wb_gemm_frac_of_nominal=fl_wb / (t_cwb - t_comb) / 1e9 / 2250.0)
         ctx.rk_poll_status()
 
     offline = None
