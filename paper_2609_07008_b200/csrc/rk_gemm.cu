@@ -36,6 +36,30 @@ struct GemmSmem {
 
 enum { WG_FULL = 31, WG_EMPTY, WG_ACC_FULL, WG_ACC_EMPTY };
 
+// Tile order.  Batched launches (head / group blocks): row block, batch, column tile, so that concurrent
+// CTAs fill whole output rows.  Single-batch launches: bands of kBandRows row blocks, inside a band column
+// tile first, then row block -- the CTAs of one wave then share kBandRows A row blocks and about
+// sm_count / kBandRows B column tiles instead of every column tile of B at once.
+constexpr int kBandRows = 16;
+__device__ __forceinline__ void tile_coords(int t, int n_tiles_m, int n_tiles_n, int n_batches, int& mb, int& batch,
+                                            int& nt) {
+  if (n_batches > 1) {
+    const int per_row_block = n_tiles_n * n_batches;
+    mb = t / per_row_block;
+    const int rem = t - mb * per_row_block;
+    batch = rem / n_tiles_n;
+    nt = rem - batch * n_tiles_n;
+    return;
+  }
+  batch = 0;
+  const int per_band = kBandRows * n_tiles_n;
+  const int band = t / per_band;
+  const int rows_here = min(kBandRows, n_tiles_m - band * kBandRows);  // the last band may be short
+  const int rem = t - band * per_band;
+  nt = rem / rows_here;
+  mb = band * kBandRows + (rem - nt * rows_here);
+}
+
 // Persistent: each CTA walks output tiles t = blockIdx.x, + gridDim.x, ... ordered row block, batch, column
 // tile (fastest), so the CTAs running at the same time cover a few 128-row blocks over the full output
 // width: they share those A rows and the whole of B through L2, and their stores fill whole output rows
@@ -95,10 +119,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) rk_gemm_kernel(const __grid_c
     uint32_t it = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-      const int mb = t / tiles_per_row_block;
-      const int rem = t - mb * tiles_per_row_block;
-      const int batch = rem / n_tiles_n;
-      const int m0 = mb * kBM, n0 = (rem % n_tiles_n) * BN;
+      int mb, batch, nt;
+      tile_coords(t, n_tiles_m, n_tiles_n, p.n_batches, mb, batch, nt);
+      const int m0 = mb * kBM, n0 = nt * BN;
       const GemmBatch bt = p.batches[batch];
       for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
         const uint32_t s = it % kStages;
@@ -166,10 +189,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) rk_gemm_kernel(const __grid_c
     if (L == 0) tma_prefetch_desc(&p.tm_c);
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
       const uint32_t b = tile_i & 1u;
-      const int mb = t / tiles_per_row_block;
-      const int rem = t - mb * tiles_per_row_block;
-      const int batch = rem / n_tiles_n;
-      const int m0 = mb * kBM, n0 = (rem % n_tiles_n) * BN;
+      int mb, batch, nt;
+      tile_coords(t, n_tiles_m, n_tiles_n, p.n_batches, mb, batch, nt);
+      const int m0 = mb * kBM, n0 = nt * BN;
       const GemmBatch bt = p.batches[batch];
       ok = mbar_wait_bounded<false>(acc_full_bar(b), (tile_i >> 1) & 1u, limit, abort_flag, p.status, WG_ACC_FULL, t);
       // the four warps leave together or not at all: the barriers below have no time limit of their own
