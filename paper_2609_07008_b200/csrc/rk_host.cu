@@ -36,7 +36,7 @@ struct rk_ctx {
   int attn_debug = 0;  // development switches of the attention kernel (rk_set_debug_flags)
   cudaStream_t copy_stream = nullptr;  // rk_layer_host: copies that overlap the kernels
   cudaStream_t copy_out_stream = nullptr;  // rk_layer_stack_host: device->host copies (full duplex with the above)
-  cudaEvent_t sev[6] = {nullptr};      // rk_layer_stack_host: in_ready[2], compute_done[2], y_copied[2]
+  cudaEvent_t sev[10] = {nullptr};     // rk_layer_stack_host: kv_ql_in[2], qg_in[2], zoff_in[2], compute_done[2], y_copied[2]
   cudaEvent_t ev[8] = {nullptr};       // device-side ordering between the two streams (no host polling)
   PFN_encodeTiled encode = nullptr;
   mutable std::string err;
@@ -233,7 +233,7 @@ rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
   ctx->n_pairs = attention_max_pairs(ctx->sm_count);
   e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_out_stream, cudaStreamNonBlocking);
-  for (int i = 0; i < 6 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->sev[i], cudaEventDisableTiming);
+  for (int i = 0; i < 10 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->sev[i], cudaEventDisableTiming);
   for (int i = 0; i < 8 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -278,7 +278,7 @@ rk_status rk_destroy(rk_ctx* ctx) {
   for (int i = 0; i < 8; ++i)
     if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
-  for (int i = 0; i < 6; ++i)
+  for (int i = 0; i < 10; ++i)
     if (ctx->sev[i]) cudaEventDestroy(ctx->sev[i]);
   if (ctx->copy_out_stream) cudaStreamDestroy(ctx->copy_out_stream);
   cudaFree(ctx->d_status);
@@ -749,6 +749,87 @@ rk_status rk_combine_offline(rk_ctx* ctx, const rk_request* rq, const void* z_on
                   ctx->prof.d_model, (int)width, ctx->off_wb, 1, st);
 }
 
+// The compute part of one layer on `st`, shared by rk_layer_host and rk_layer_stack_host.  Inputs may still
+// be on their way: ev_ql_rest (NULL = none) guards the protected-row queries beyond the request's first
+// Local range, ev_qg the Global queries, ev_zoff the artifact.  With split_global the Global pass and
+// everything after it run in the request's two row ranges; the y rows of each range are copied to the
+// host on y_stream as soon as they are complete (chunk_ev: two events that order those copies).
+static rk_status layer_compute(rk_ctx* ctx, const rk_request* rq, const rk_layer_buffers* dev, const void* W_uv,
+                               const void* W_a, const void* W_b, cudaStream_t st, cudaEvent_t ev_ql_rest, cudaEvent_t ev_qg,
+                               cudaEvent_t ev_zoff, bool split_global, void* y_host, cudaStream_t y_stream,
+                               cudaEvent_t* chunk_ev) {
+  const int G = ctx->prof.n_groups, H = ctx->prof.n_heads, L = H - G, ro = ctx->prof.o_rank;
+  const int64_t T = rq->T, dm = ctx->prof.d_model;
+  const size_t width = (size_t)G * ro;
+  const bool has_l = rq->A > 0;
+  if (!aligned16(dev->kv) || !aligned16(dev->q_g) || !aligned16(dev->O_g) || !aligned16(dev->z_on_g) || !aligned16(dev->z) ||
+      !aligned16(dev->y) || (reinterpret_cast<uintptr_t>(dev->workspace) & 255u))
+    return fail(ctx, RK_ERR_ALIGN, "device buffers must be 16-byte aligned and the workspace 256-byte aligned");
+  if (dev->workspace_bytes < proj_ws_bytes(rq)) return fail(ctx, RK_ERR_WORKSPACE, "workspace too small: need %zu bytes", proj_ws_bytes(rq));
+  cudaError_t e = cudaSuccess;
+  rk_status s = RK_OK;
+  if (has_l) {  // Local pass and the Local half of the first projection: need kv, q_l only
+    if (!aligned16(dev->q_l) || !aligned16(dev->O_l)) return fail(ctx, RK_ERR_ALIGN, "device buffers must be 16-byte aligned");
+    if (ev_ql_rest != nullptr && rq->split_slot > 0) {
+      s = attn_pass(ctx, rq, dev->kv, dev->q_l, rq->A, L, rq->d_prot_rows, rq->d_work_l_part[0], rq->n_tiles_l_part[0],
+                    dev->O_l, dev->lse_l, st);
+      e = cudaStreamWaitEvent(st, ev_ql_rest, 0);
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
+      if (s == RK_OK)
+        s = attn_pass(ctx, rq, dev->kv, dev->q_l, rq->A, L, rq->d_prot_rows, rq->d_work_l_part[1], rq->n_tiles_l_part[1],
+                      dev->O_l, dev->lse_l, st);
+    } else {
+      s = attn_pass(ctx, rq, dev->kv, dev->q_l, rq->A, L, rq->d_prot_rows, rq->d_work_l, rq->n_tiles_l, dev->O_l,
+                    dev->lse_l, st);
+    }
+    if (s == RK_OK)
+      s = rk_group_sliced_proj(ctx, rq, nullptr, dev->O_l, W_uv, W_a, nullptr, dev->z_on_l, dev->workspace,
+                               dev->workspace_bytes, st);
+    if (s != RK_OK) return s;
+  }
+  e = cudaStreamWaitEvent(st, ev_qg, 0);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
+  // Global pass, Global half of the first projection, restore-and-replace and W_b per row range; the y
+  // rows of a range are copied out while the next range computes
+  const int n_chunks = (split_global && rq->split_tok > 0) ? 2 : 1;
+  const uint8_t* Og = reinterpret_cast<const uint8_t*>(dev->O_g);
+  uint8_t* og = reinterpret_cast<uint8_t*>(dev->workspace);  // per-head W_uv output of the Global heads
+  uint8_t* zg = reinterpret_cast<uint8_t*>(dev->z_on_g);
+  const uint8_t* zo = reinterpret_cast<const uint8_t*>(dev->z_off);
+  uint8_t* zz = reinterpret_cast<uint8_t*>(dev->z);
+  uint8_t* yy = reinterpret_cast<uint8_t*>(dev->y);
+  for (int c = 0; c < n_chunks; ++c) {
+    const int64_t r0 = c == 0 ? 0 : rq->split_tok, r1 = (n_chunks == 2 && c == 0) ? rq->split_tok : T;
+    const int64_t n = r1 - r0;
+    s = attn_pass(ctx, rq, dev->kv, dev->q_g, T, G, nullptr, n_chunks == 2 ? rq->d_work_g_part[c] : rq->d_work_g,
+                  n_chunks == 2 ? rq->n_tiles_g_part[c] : rq->n_tiles_g, dev->O_g, dev->lse_g, st);
+    if (s == RK_OK)
+      s = run_gemm(ctx, Og + (size_t)r0 * G * kDLatent * 2, n, (int64_t)G * kDLatent, W_uv, (int64_t)H * kDV, kDLatent,
+                   og + (size_t)r0 * G * kDV * 2, (int64_t)G * kDV, (int)n, kDV, kDLatent, ctx->off_uv_g, G, st);
+    if (s == RK_OK)
+      s = run_gemm(ctx, og + (size_t)r0 * G * kDV * 2, n, (int64_t)G * kDV, W_a, (int64_t)G * ro, kGroup * kDV,
+                   zg + (size_t)r0 * width * 2, (int64_t)G * ro, (int)n, ro, kDV, ctx->off_wa_g, G, st);
+    if (s != RK_OK) return s;
+    if (c == 0) {  // the artifact has to be there from here on
+      e = cudaStreamWaitEvent(st, ev_zoff, 0);
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
+    }
+    e = launch_combine(zg + (size_t)r0 * width * 2, dev->z_on_l, zo ? zo + (size_t)r0 * width * 2 : nullptr, rq->d_inv_map + r0, n,
+                       (int64_t)width, zz + (size_t)r0 * width * 2, ctx->sm_count, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "combine launch");
+    s = run_gemm(ctx, zz + (size_t)r0 * width * 2, n, (int64_t)width, W_b, dm, (int64_t)width, yy + (size_t)r0 * dm * 2, dm, (int)n,
+                 (int)dm, (int)width, ctx->off_wb, 1, st);
+    if (s != RK_OK) return s;
+    e = cudaEventRecord(chunk_ev[c], st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(y_stream, chunk_ev[c], 0);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(reinterpret_cast<uint8_t*>(y_host) + (size_t)r0 * dm * 2, yy + (size_t)r0 * dm * 2, (size_t)n * dm * 2,
+                          cudaMemcpyDeviceToHost, y_stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "device to host copy");
+  }
+  return RK_OK;
+}
+
 rk_status rk_layer_host(rk_ctx* ctx, const rk_request* rq, const void* kv_host, const void* q_g_host,
                         const void* q_l_host, const void* z_off_host, const void* W_uv, const void* W_a,
                         const void* W_b, const rk_layer_buffers* dev, void* y_host, void* stream) {
@@ -787,71 +868,9 @@ rk_status rk_layer_host(rk_ctx* ctx, const rk_request* rq, const void* kv_host, 
     e = cudaMemcpyAsync(dev->z_off, z_off_host, (size_t)rq->n_off_rows * width * 2, cudaMemcpyHostToDevice, cp);
   if (e == cudaSuccess) e = cudaEventRecord(ctx->ev[2], cp);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "host to device copy");
-  if (!aligned16(dev->kv) || !aligned16(dev->q_g) || !aligned16(dev->O_g) || !aligned16(dev->z_on_g) || !aligned16(dev->z) ||
-      !aligned16(dev->y) || (reinterpret_cast<uintptr_t>(dev->workspace) & 255u))
-    return fail(ctx, RK_ERR_ALIGN, "device buffers must be 16-byte aligned and the workspace 256-byte aligned");
-  if (dev->workspace_bytes < proj_ws_bytes(rq)) return fail(ctx, RK_ERR_WORKSPACE, "workspace too small: need %zu bytes", proj_ws_bytes(rq));
-  const int H = ctx->prof.n_heads, ro = ctx->prof.o_rank;
-  rk_status s = RK_OK;
-  if (has_l) {  // Local pass and the Local half of the first projection: need kv, q_l only
-    if (!aligned16(dev->q_l) || !aligned16(dev->O_l)) return fail(ctx, RK_ERR_ALIGN, "device buffers must be 16-byte aligned");
-    if (slot0 < rq->A) {
-      s = attn_pass(ctx, rq, dev->kv, dev->q_l, rq->A, L, rq->d_prot_rows, rq->d_work_l_part[0], rq->n_tiles_l_part[0],
-                    dev->O_l, dev->lse_l, st);
-      e = cudaStreamWaitEvent(st, ctx->ev[6], 0);
-      if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
-      if (s == RK_OK)
-        s = attn_pass(ctx, rq, dev->kv, dev->q_l, rq->A, L, rq->d_prot_rows, rq->d_work_l_part[1], rq->n_tiles_l_part[1],
-                      dev->O_l, dev->lse_l, st);
-    } else {
-      s = attn_pass(ctx, rq, dev->kv, dev->q_l, rq->A, L, rq->d_prot_rows, rq->d_work_l, rq->n_tiles_l, dev->O_l,
-                    dev->lse_l, st);
-    }
-    if (s == RK_OK)
-      s = rk_group_sliced_proj(ctx, rq, nullptr, dev->O_l, W_uv, W_a, nullptr, dev->z_on_l, dev->workspace,
-                               dev->workspace_bytes, stream);
-    if (s != RK_OK) return s;
-  }
-  e = cudaStreamWaitEvent(st, ctx->ev[1], 0);
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
-  // Global pass, Global half of the first projection, restore-and-replace and W_b per row range; the y
-  // rows of a range are copied out while the next range computes
-  const int n_chunks = rq->split_tok > 0 ? 2 : 1;
-  const uint8_t* Og = reinterpret_cast<const uint8_t*>(dev->O_g);
-  uint8_t* og = reinterpret_cast<uint8_t*>(dev->workspace);  // per-head W_uv output of the Global heads
-  uint8_t* zg = reinterpret_cast<uint8_t*>(dev->z_on_g);
-  const uint8_t* zo = reinterpret_cast<const uint8_t*>(dev->z_off);
-  uint8_t* zz = reinterpret_cast<uint8_t*>(dev->z);
-  uint8_t* yy = reinterpret_cast<uint8_t*>(dev->y);
-  for (int c = 0; c < n_chunks; ++c) {
-    const int64_t r0 = c == 0 ? 0 : rq->split_tok, r1 = (n_chunks == 2 && c == 0) ? rq->split_tok : T;
-    const int64_t n = r1 - r0;
-    s = attn_pass(ctx, rq, dev->kv, dev->q_g, T, G, nullptr, n_chunks == 2 ? rq->d_work_g_part[c] : rq->d_work_g,
-                  n_chunks == 2 ? rq->n_tiles_g_part[c] : rq->n_tiles_g, dev->O_g, dev->lse_g, st);
-    if (s == RK_OK)
-      s = run_gemm(ctx, Og + (size_t)r0 * G * kDLatent * 2, n, (int64_t)G * kDLatent, W_uv, (int64_t)H * kDV, kDLatent,
-                   og + (size_t)r0 * G * kDV * 2, (int64_t)G * kDV, (int)n, kDV, kDLatent, ctx->off_uv_g, G, st);
-    if (s == RK_OK)
-      s = run_gemm(ctx, og + (size_t)r0 * G * kDV * 2, n, (int64_t)G * kDV, W_a, (int64_t)G * ro, kGroup * kDV,
-                   zg + (size_t)r0 * width * 2, (int64_t)G * ro, (int)n, ro, kDV, ctx->off_wa_g, G, st);
-    if (s != RK_OK) return s;
-    if (c == 0) {  // the artifact has to be there from here on
-      e = cudaStreamWaitEvent(st, ctx->ev[2], 0);
-      if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
-    }
-    e = launch_combine(zg + (size_t)r0 * width * 2, dev->z_on_l, zo ? zo + (size_t)r0 * width * 2 : nullptr, rq->d_inv_map + r0, n,
-                       (int64_t)width, zz + (size_t)r0 * width * 2, ctx->sm_count, st);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "combine launch");
-    s = run_gemm(ctx, zz + (size_t)r0 * width * 2, n, (int64_t)width, W_b, dm, (int64_t)width, yy + (size_t)r0 * dm * 2, dm, (int)n,
-                 (int)dm, (int)width, ctx->off_wb, 1, st);
-    if (s != RK_OK) return s;
-    e = cudaEventRecord(ctx->ev[3 + c], st);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(cp, ctx->ev[3 + c], 0);
-    if (e == cudaSuccess)
-      e = cudaMemcpyAsync(reinterpret_cast<uint8_t*>(y_host) + (size_t)r0 * dm * 2, yy + (size_t)r0 * dm * 2, (size_t)n * dm * 2,
-                          cudaMemcpyDeviceToHost, cp);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "device to host copy");
-  }
+  rk_status s = layer_compute(ctx, rq, dev, W_uv, W_a, W_b, st, slot0 < rq->A ? ctx->ev[6] : nullptr, ctx->ev[1], ctx->ev[2],
+                              rq->split_tok > 0, y_host, cp, &ctx->ev[3]);
+  if (s != RK_OK) return s;
   e = cudaEventRecord(ctx->ev[7], cp);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(st, ctx->ev[7], 0);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -873,24 +892,29 @@ rk_status rk_layer_stack_host(rk_ctx* ctx, int32_t n_layers, const rk_layer_io* 
   }
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   cudaStream_t cin = ctx->copy_stream, cout = ctx->copy_out_stream;
-  cudaEvent_t* in_ready = ctx->sev;          // [2] inputs of buffer set b are on the device
-  cudaEvent_t* compute_done = ctx->sev + 2;  // [2] the layer running on set b has finished
-  cudaEvent_t* y_copied = ctx->sev + 4;      // [2] y of the layer that ran on set b is on the host
+  cudaEvent_t* kv_ql_in = ctx->sev;          // [2] kv and q_l of buffer set b are on the device
+  cudaEvent_t* qg_in = ctx->sev + 2;         // [2] ... q_g
+  cudaEvent_t* zoff_in = ctx->sev + 4;       // [2] ... the artifact
+  cudaEvent_t* compute_done = ctx->sev + 6;  // [2] the layer running on set b has finished
+  cudaEvent_t* y_copied = ctx->sev + 8;      // [2] y of the layer that ran on set b is on the host
   const rk_layer_buffers* sets[2] = {dev0, dev1};
   const int G = ctx->prof.n_groups, L = ctx->prof.n_heads - G;
   const size_t width = (size_t)G * ctx->prof.o_rank;
 
-  auto copy_in = [&](int l) -> cudaError_t {  // host -> device of layer l into set l & 1, on the copy-in stream
+  // host -> device of layer l into set l & 1, on the copy-in stream, in the order the layer consumes them
+  auto copy_in = [&](int l) -> cudaError_t {
     const rk_layer_io& io = layers[l];
     const rk_request* rq = io.req;
     const rk_layer_buffers* d = sets[l & 1];
     cudaError_t e = cudaMemcpyAsync(d->kv, io.kv_host, (size_t)rq->T * kDQK * 2, cudaMemcpyHostToDevice, cin);
     if (e == cudaSuccess && rq->A > 0)
       e = cudaMemcpyAsync(d->q_l, io.q_l_host, (size_t)rq->A * L * kDQK * 2, cudaMemcpyHostToDevice, cin);
+    if (e == cudaSuccess) e = cudaEventRecord(kv_ql_in[l & 1], cin);
     if (e == cudaSuccess) e = cudaMemcpyAsync(d->q_g, io.q_g_host, (size_t)rq->T * G * kDQK * 2, cudaMemcpyHostToDevice, cin);
+    if (e == cudaSuccess) e = cudaEventRecord(qg_in[l & 1], cin);
     if (e == cudaSuccess && rq->n_off_rows > 0 && io.z_off_host)
       e = cudaMemcpyAsync(d->z_off, io.z_off_host, (size_t)rq->n_off_rows * width * 2, cudaMemcpyHostToDevice, cin);
-    if (e == cudaSuccess) e = cudaEventRecord(in_ready[l & 1], cin);
+    if (e == cudaSuccess) e = cudaEventRecord(zoff_in[l & 1], cin);
     return e;
   };
 
@@ -903,28 +927,21 @@ rk_status rk_layer_stack_host(rk_ctx* ctx, int32_t n_layers, const rk_layer_io* 
   for (int l = 0; l < n_layers; ++l) {
     const int b = l & 1;
     const rk_layer_io& io = layers[l];
-    const rk_request* rq = io.req;
     const rk_layer_buffers* d = sets[b];
-    const bool has_l = rq->A > 0;
     if (l + 1 < n_layers) {  // prefetch the next layer while this one computes
       if (l >= 1) e = cudaStreamWaitEvent(cin, compute_done[b ^ 1], 0);  // layer l-1 has released set b^1
       if (e == cudaSuccess) e = copy_in(l + 1);
       if (e != cudaSuccess) return cuda_fail(ctx, e, "host to device copy");
     }
-    e = cudaStreamWaitEvent(st, in_ready[b], 0);
+    e = cudaStreamWaitEvent(st, kv_ql_in[b], 0);
     if (e == cudaSuccess && l >= 2) e = cudaStreamWaitEvent(st, y_copied[b], 0);  // y of layer l-2 has left set b
     if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
-    rk_status s = rk_mla_online_attn(ctx, rq, d->kv, d->q_g, has_l ? d->q_l : nullptr, d->O_g, d->lse_g,
-                                     has_l ? d->O_l : nullptr, has_l ? d->lse_l : nullptr, stream);
-    if (s == RK_OK)
-      s = rk_group_sliced_proj(ctx, rq, d->O_g, has_l ? d->O_l : nullptr, io.W_uv, io.W_a, d->z_on_g,
-                               has_l ? d->z_on_l : nullptr, d->workspace, d->workspace_bytes, stream);
-    if (s == RK_OK) s = rk_combine_offline(ctx, rq, d->z_on_g, d->z_on_l, d->z_off, io.W_b, d->z, d->y, stream);
+    // the first layer starts as soon as its first inputs are in; the last layer returns y in two row
+    // ranges so that only the second one's copy is left when the kernels end
+    rk_status s = layer_compute(ctx, io.req, d, io.W_uv, io.W_a, io.W_b, st, nullptr, qg_in[b], zoff_in[b],
+                                l == n_layers - 1, io.y_host, cout, &ctx->ev[3]);
     if (s != RK_OK) return s;
     e = cudaEventRecord(compute_done[b], st);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(cout, compute_done[b], 0);
-    if (e == cudaSuccess)
-      e = cudaMemcpyAsync(io.y_host, d->y, (size_t)rq->T * ctx->prof.d_model * 2, cudaMemcpyDeviceToHost, cout);
     if (e == cudaSuccess) e = cudaEventRecord(y_copied[b], cout);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "device to host copy");
   }
