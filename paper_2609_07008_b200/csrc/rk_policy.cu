@@ -93,12 +93,16 @@ __global__ void __launch_bounds__(kPolicyThreads) policy_select_kernel(PolicyPar
   if (threadIdx.x < 256) hist[threadIdx.x] = 0u;
   __syncthreads();
   const int t = blockIdx.x * kPolicyThreads + threadIdx.x;
+  unsigned bin = 0xffffffffu;  // not counted
   if (t < p.T && (p.flags[t] & (kPolicyStructural | kPolicyCandidate)) == kPolicyCandidate) {
     const unsigned long long key = select_key(p.scores[t], t);
     const unsigned long long prefix = p.state->prefix;
     const bool match = (d == 7) || ((key >> (8 * (d + 1))) == (prefix >> (8 * (d + 1))));
-    if (match) atomicAdd(&hist[(unsigned)(key >> (8 * d)) & 255u], 1u);
+    if (match) bin = (unsigned)(key >> (8 * d)) & 255u;
   }
+  // scores cluster in a few exponent bins: one shared-memory atomic per distinct bin of a warp
+  const unsigned peers = __match_any_sync(0xffffffffu, bin);
+  if (bin != 0xffffffffu && (threadIdx.x & 31) == (unsigned)(__ffs(peers) - 1)) atomicAdd(&hist[bin], (unsigned)__popc(peers));
   __syncthreads();
   if (threadIdx.x < 256 && hist[threadIdx.x] != 0u) atomicAdd(&p.state->hist[threadIdx.x], hist[threadIdx.x]);
   __threadfence();
