@@ -180,6 +180,10 @@ CONFIGS = {
     "flash32k":  dict(H=64,  G=8,  docs="u16",       shuffle=True,  n_q=2048, pct_bp=None, run_len=1, r_o=1024, d_model=4096, seed=2),
     "flash256k": dict(H=64,  G=8,  docs=[4096] * 64, shuffle=True,  n_q=2048, pct_bp=200, run_len=16, r_o=1024, d_model=4096, seed=3),
     "pro128k":   dict(H=128, G=16, docs=[4096] * 32, shuffle=True,  n_q=4096, pct_bp=300, run_len=1,  r_o=1024, d_model=7168, seed=4),
+    # not one of the five benchmark shapes: the longest context the paper's length table names (440K), with ragged
+    # document lengths, as a parity case for long requests
+    "flash440k": dict(H=64,  G=8,  docs=[4096] * 100 + [3000, 4500, 5000, 2999, 7777, 4100], shuffle=True, n_q=2048,
+                      pct_bp=200, run_len=16, r_o=1024, d_model=4096, seed=5),
 }
 N_LAYERS_FLASH32K = 37
 

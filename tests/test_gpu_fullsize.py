@@ -47,7 +47,7 @@ def sample_within_budget(w, budget_pairs, n_random=24):
 
 @pytest.mark.parametrize("name, regime, budget", [
     ("flash1", "mandated", 4e7), ("flash1", "sharp", 4e7), ("flash32k", "mandated", 4e7),
-    ("flash256k", "mandated", 6e7), ("pro128k", "mandated", 6e7),
+    ("flash256k", "mandated", 6e7), ("pro128k", "mandated", 6e7), ("flash440k", "mandated", 8e7),
 ])
 def test_full_size_layer_on_sampled_rows(rk, name, regime, budget):
     """Whole layer (the three calls bench.py times) at full size; sampled rows against the checker."""
