@@ -332,6 +332,10 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     rkdist.init("nccl", dev)
+    from paper_2609_07008_b200 import build as rkbuild
+    if local_rank == 0:
+        rkbuild.ensure_built()                        # a fresh checkout: compile once with nvcc (no other path exists)
+    rkdist.barrier()
     from paper_2609_07008_b200 import binding as rk   # raises if librk.so is missing: no fallback
 
     name = args.config

@@ -63,5 +63,11 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     return LIB_PATH
 
 
+def ensure_built() -> str:
+    """Builds the library if the built file is not there (a fresh checkout); an existing build is left alone.
+    A missing compiler is an error: nothing else can compute the path."""
+    return LIB_PATH if os.path.exists(LIB_PATH) else build_library(force=True)
+
+
 if __name__ == "__main__":
     print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))

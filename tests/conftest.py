@@ -24,3 +24,10 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library_is_built():
+    """A fresh checkout has no built library (it is kept out of the history): build it once, with nvcc."""
+    from paper_2609_07008_b200 import build
+    build.ensure_built()
