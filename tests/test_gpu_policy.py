@@ -9,7 +9,7 @@ import torch
 
 from oracle import policy
 from paper_2609_07008_b200 import synth
-from tests.test_oracle_policy_pins import read_example
+from tests.test_oracle_policy_pins import read_example, read_moe_examples
 
 pytestmark = pytest.mark.gpu
 
@@ -127,6 +127,12 @@ def test_moe_fanout_matches_checker(ctx, tau):
     ctx.rk_poll_status()
     assert np.array_equal(k.cpu().numpy(), k_want)
     assert np.array_equal(keep.cpu().numpy(), keep_want)
+
+
+def test_moe_hand_worked_examples(ctx):
+    for w, tau, k_want, kept in read_moe_examples():
+        k, keep = ctx.rk_moe_fanout(torch.tensor([w], dtype=torch.float32, device="cuda"), tau)
+        assert int(k[0]) == k_want and [s for s in range(6) if (int(keep[0]) >> s) & 1] == kept, (w, tau)
 
 
 def test_moe_fanout_edge_cases(ctx):

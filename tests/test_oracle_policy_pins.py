@@ -9,6 +9,18 @@ import pytest
 from oracle import policy
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "protected_rows_example.txt")
+GOLDEN_MOE = os.path.join(os.path.dirname(__file__), "golden", "moe_fanout_example.txt")
+
+
+def read_moe_examples():
+    cases = []
+    for line in open(GOLDEN_MOE):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        w, tau, k, kept = [f.strip() for f in line.split("|")]
+        cases.append(([float(x) for x in w.split()], float(tau), int(k), [int(x) for x in kept.split()]))
+    return cases
 
 
 def read_example():
@@ -116,6 +128,15 @@ def test_budget_identity_and_top_up_order(bp):
         worst_in = min((float(scores[t]), -t) for t in added)
         best_out = max((float(scores[t]), -t) for t in left)
         assert worst_in > best_out
+
+
+def test_moe_hand_worked_examples():
+    cases = read_moe_examples()
+    assert len(cases) == 12
+    for w, tau, k_want, kept in cases:
+        k, keep = policy.moe_fanout(np.array([w], dtype=np.float32), tau)
+        assert int(k[0]) == k_want, (w, tau)
+        assert [s for s in range(6) if (int(keep[0]) >> s) & 1] == kept, (w, tau)
 
 
 def test_moe_geometric_weights_closed_form():
