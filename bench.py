@@ -497,7 +497,7 @@ def main():
     rest_tflops = (fl_proj + fl_wb) / (np.mean(rest_ms) * 1e-3) / 1e12
 
     cpu_baseline = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:   # the checker is timed at N = 1 only
         run_layer(w, req)                      # leave layer 0's y in the buffer for the parity figure below
         torch.cuda.synchronize()
         rows = pick_oracle_rows(w, args.oracle_pairs)
