@@ -91,7 +91,7 @@ cudaError_t launch_combine(const void* z_on_g, const void* z_on_l, const void* z
 constexpr uint8_t kPolicyStructural = 1, kPolicyCandidate = 2, kPolicyDirty = 4;
 
 struct PolicyState {
-  unsigned n_cand, n_struct_cand, blocks_done, n_top, k_rem, pad;
+  unsigned n_cand, n_struct_cand, blocks_done, n_top, k_rem, done;
   unsigned long long prefix;  // digits of the n_top-th largest (score,row) key found so far
   unsigned hist[256];
 };

@@ -87,7 +87,9 @@ __global__ void __launch_bounds__(kPolicyThreads) policy_flags_kernel(PolicyPara
 // rows whose higher digits equal the prefix found so far; the last block to finish picks the digit
 // that holds the k_rem-th largest key and leaves the histogram clean for the next pass.
 __global__ void __launch_bounds__(kPolicyThreads) policy_select_kernel(PolicyParams p, int d) {
-  if (*(volatile unsigned*)&p.state->n_top == 0u) return;
+  // nothing to pick, or an earlier digit already ended the search (its whole bin was needed, so the
+  // prefix with zeros below it is the threshold)
+  if (*(volatile unsigned*)&p.state->n_top == 0u || *(volatile unsigned*)&p.state->done != 0u) return;
   __shared__ unsigned hist[256];
   __shared__ bool last;
   if (threadIdx.x < 256) hist[threadIdx.x] = 0u;
@@ -121,6 +123,7 @@ __global__ void __launch_bounds__(kPolicyThreads) policy_select_kernel(PolicyPar
     }
     p.state->k_rem = k - above;
     p.state->prefix |= (unsigned long long)digit << (8 * d);
+    if (above + gh[digit] == k) p.state->done = 1u;
     for (int b = 0; b < 256; ++b) gh[b] = 0u;
     p.state->blocks_done = 0u;
   }
