@@ -315,6 +315,9 @@ def main():
                     help="visible-pair budget of the CPU checker sample (about 10-30 s of host work)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--protect-bp", type=int, default=None,
+                    help="override the share of protected document rows (basis points), e.g. the paper's controller "
+                         "budgets 1000 / 2000 / 2500; default: the configuration's own share")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-aux", action="store_true", help="skip the standalone relocation / merge timings")
     ap.add_argument("--with-offline", action="store_true", help="also time the offline artifact build")
@@ -343,7 +346,7 @@ def main():
     ctx = None
     layers = []          # (workload, request) per layer: same layout, own values, own protected rows
     for l in range(n_layers):
-        prof, lay, prot = synth.make_geometry(name, layer=l)
+        prof, lay, prot = synth.make_geometry(name, layer=l, pct_bp=args.protect_bp)
         # every rank gets its own request values (independent requests, same shape)
         wl = synth.make_tensors(name, prof, lay, prot, rkdist.rank_seed(synth.CONFIGS[name]["seed"], rank) + 7 * l,
                                 device=dev, regime=args.regime)

@@ -188,10 +188,11 @@ CONFIGS = {
 N_LAYERS_FLASH32K = 37
 
 
-def make_geometry(name: str, layer: int = 0, seed: Optional[int] = None):
+def make_geometry(name: str, layer: int = 0, seed: Optional[int] = None, pct_bp: Optional[int] = None):
     """Returns (profile, layout, prot_rows) for a named configuration.  For 'flash32k'
     every layer shares the layout (one request) but draws its own protected rows with a
-    fraction uniform in [2 %, 5 %]."""
+    fraction uniform in [2 %, 5 %].  pct_bp overrides the configuration's protected share
+    (basis points of the document rows), e.g. the controller budgets 1000 / 2000 / 2500."""
     cfg = CONFIGS[name]
     seed = cfg["seed"] if seed is None else seed
     rng = np.random.default_rng(np.random.PCG64(seed))
@@ -200,7 +201,8 @@ def make_geometry(name: str, layer: int = 0, seed: Optional[int] = None):
         docs = rng.integers(1024, 4097, size=16).tolist()
     layout = make_layout(docs, cfg["n_q"], rng, cfg["shuffle"])
     gh = draw_global_heads(cfg["G"], rng)
-    pct_bp = cfg["pct_bp"]
+    override = pct_bp
+    pct_bp = cfg["pct_bp"] if override is None else int(override)
     rng_rows = rng
     if pct_bp is None:
         rng_rows = np.random.default_rng(np.random.PCG64(seed * 1000 + layer))
