@@ -314,6 +314,14 @@ def test_no_protected_rows(rk):
     exp = oracle_online(w, np.arange(lay.n_rows))
     y = _layer(rk, w)
     assert_close(f64(y), exp["y"], "y")
+    # the host-buffer entry point without any Local work (no q_l at all)
+    ctx, req = make(rk, w)
+    bufs = ctx.alloc_layer_buffers(req, "cuda")
+    pin = lambda t: t.cpu().pin_memory()
+    y_h = torch.empty((lay.n_rows, prof.d_model), dtype=torch.bfloat16).pin_memory()
+    ctx.rk_layer_host(req, pin(w.kv), pin(w.q_g), None, pin(w.z_off), w.w_uv, w.w_a, w.w_b, bufs, y_h)
+    ctx.rk_poll_status()
+    assert torch.equal(y_h, y.cpu())
 
 
 def test_gaps_between_segments_and_large_offsets(rk):
