@@ -104,20 +104,20 @@ struct SegIter {
       int lo = 0, hi = p.n_segs - 1;
       while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
-        if (__ldg(p.seg_off + mid) <= prow0) lo = mid; else hi = mid - 1;
+        if (p.seg_off[mid] <= prow0) lo = mid; else hi = mid - 1;
       }
       seg = lo - 1;
     }
   }
   __device__ bool next() {
     while (++seg < p.n_segs) {
-      const int lo = __ldg(p.seg_off + seg), hi = __ldg(p.seg_off + seg + 1);
+      const int lo = p.seg_off[seg], hi = p.seg_off[seg + 1];
       if (p.isolated) {
         if (lo > prow1) { seg = p.n_segs; return false; }  // past the tile's last row: nothing further overlaps
         if (prow1 < lo || prow0 >= hi) { kmax = 0; continue; }
         kmax = (prow1 < hi ? prow1 : hi - 1) - lo + 1;
       } else {
-        const int lim = maxpos - __ldg(p.seg_delta + seg) + 1;
+        const int lim = maxpos - p.seg_delta[seg] + 1;
         kmax = lim < hi - lo ? lim : hi - lo;
       }
       if (kmax > 0) return true;
@@ -351,7 +351,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       SegIter it(p, item);
       int prev_row0 = -1, prev_kb = 0;
       while (ok && it.next()) {
-        const int row0 = __ldg(p.seg_off + it.seg);
+        const int row0 = p.seg_off[it.seg];
         for (int kb = 0; kb < it.kmax && ok; kb += kAttnKeysPerTile) {
           ok = load_k(row0, kb, w);
           if (ok && prev_row0 >= 0) ok = load_v(prev_row0, prev_kb, w);
@@ -620,35 +620,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     const uint32_t s_free_remote = mapa_shared(bar(kBarSFree), 0);
     const uint32_t qh_done_remote = mapa_shared(bar(kBarQhDone), 0);
 
-    // Moves this thread's share of the upper Q half of row tile w_next (row m, 64 dims) from its ring
-    // stage into tensor memory.  Called once the QK^T MMAs that read the previous contents are complete:
-    // before the first row tile, and afterwards between the last PV of a row tile and that tile's
-    // epilogue, so that the next tile's first QK^T runs under the epilogue.
-    auto move_q_upper = [&](int w_next) -> bool {
-      if (!mbar_wait_bounded<false>(bar(kBarQhFull), qh_full_phase, limit, abort_flag, p.status, W_QHFULL, w_next))
-        return false;
-      qh_full_phase ^= 1;
-      // every role counts ring positions alike: one staged half per row tile, nine stages per key tile
-      const uint8_t* stage = smem + kOffRing + (ring_it % kStages) * kStageBytes;
-      ring_it += 1u + 9u * (uint32_t)count_key_tiles(p, get_work(p, w_next));
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t qv[32];
-        const uint8_t* chunk = stage + (2 * ch + half) * kQChunkBytes;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint4 v = *reinterpret_cast<const uint4*>(chunk + sw128_offset((uint32_t)m, (uint32_t)c));
-          qv[4 * c] = v.x; qv[4 * c + 1] = v.y; qv[4 * c + 2] = v.z; qv[4 * c + 3] = v.w;
-        }
-        tmem_st_x32(tmem_base + lane_base + kColQ + (uint32_t)(ch * 64 + half * 32), qv);
-      }
-      tmem_wait_st();
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_remote(qh_done_remote);
-      return true;
-    };
-
     for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
       const AttnWorkItem item = get_work(p, w);
       const int r = item.tile * kAttnRowsPerPair + (int)crank * kAttnRowsPerCta + m;
@@ -661,17 +632,38 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       }
       float m_run = -INFINITY, l_run = 0.f;
       int kt = 0;
-      if (w == pair) ok = move_q_upper(w);  // later row tiles: done before the previous tile's epilogue
-      if (!ok) break;
+      {  // move this thread's share of the upper Q half (row m, 64 dims) from its ring stage into TMEM
+        ok = mbar_wait_bounded<false>(bar(kBarQhFull), qh_full_phase, limit, abort_flag, p.status, W_QHFULL, w);
+        qh_full_phase ^= 1;
+        if (!ok) break;
+        // every role counts ring positions alike: one staged half per row tile, nine stages per key tile
+        const uint8_t* stage = smem + kOffRing + (ring_it % kStages) * kStageBytes;
+        ring_it += 1u + 9u * (uint32_t)count_key_tiles(p, item);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t qv[32];
+          const uint8_t* chunk = stage + (2 * ch + half) * kQChunkBytes;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint4 v = *reinterpret_cast<const uint4*>(chunk + sw128_offset((uint32_t)m, (uint32_t)c));
+            qv[4 * c] = v.x; qv[4 * c + 1] = v.y; qv[4 * c + 2] = v.z; qv[4 * c + 3] = v.w;
+          }
+          tmem_st_x32(tmem_base + lane_base + kColQ + (uint32_t)(ch * 64 + half * 32), qv);
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_remote(qh_done_remote);
+      }
 
       SegIter it(p, item);
       while (ok && it.next()) {
-        const int n_seg = __ldg(p.seg_off + it.seg + 1) - __ldg(p.seg_off + it.seg);
-        int lim = pos - __ldg(p.seg_delta + it.seg);  // last visible canonical index
+        const int n_seg = p.seg_off[it.seg + 1] - p.seg_off[it.seg];
+        int lim = pos - p.seg_delta[it.seg];  // last visible canonical index
         if (lim > n_seg - 1) lim = n_seg - 1;
         if (pos < 0) lim = -1;
         if (p.isolated) {  // only the row's own segment, causal in its canonical frame
-          const int lo = __ldg(p.seg_off + it.seg);
+          const int lo = p.seg_off[it.seg];
           lim = (prow >= lo && prow < lo + n_seg) ? prow - lo : -1;
         }
         for (int kb = 0; kb < it.kmax && ok; kb += kAttnKeysPerTile, ++kt) {
@@ -802,11 +794,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       pv_done_phase ^= 1;
       if (!ok) break;
       tc_fence_after_sync();
-      // every MMA of this row tile is complete: the next tile's upper Q half may replace this one's
-      if (w + p.n_pairs < p.n_tiles) {
-        ok = move_q_upper(w + p.n_pairs);
-        if (!ok) break;
-      }
       float l_tot = l_run;
       ok = quad_exchange_sum(xbuf, part, m, ++xseq, l_run, l_tot, limit, abort_flag, p.status, w);
       if (!ok) break;
