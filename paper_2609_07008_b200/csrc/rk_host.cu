@@ -841,7 +841,7 @@ rk_status rk_layer_host(rk_ctx* ctx, const rk_request* rq, const void* kv_host, 
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   cudaStream_t cp = ctx->copy_stream;
   const int G = ctx->prof.n_groups, L = ctx->prof.n_heads - G;
-  const int64_t T = rq->T, dm = ctx->prof.d_model;
+  const int64_t T = rq->T;
   const size_t width = (size_t)G * ctx->prof.o_rank;
   const bool has_l = rq->A > 0;
   // The copy stream starts after everything already queued on `stream` (the staging buffers may
