@@ -19,4 +19,5 @@ artifacts is from full recomputation on random data) -- the paper quantifies tha
 through model-level F1/EM, so there is nothing to pin it to.
 """
 from .mla_online import *  # noqa: F401,F403
+from . import phase  # noqa: F401  (output-phase variant: RestorePhase / R^{-1}; pins in tests/test_oracle_phase_pins.py)
 from . import policy  # noqa: F401  (Eq. protected and Eq. moe; pins in tests/test_oracle_policy_pins.py)
