@@ -7,9 +7,11 @@ rk_combine_offline (restore-and-replace + shared W_b).  Metric: prefill tokens/s
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
 
-With N > 1 (launched by torch.distributed.run) every rank runs its own independent request of
-the same shape (the path has no exchange step: weak scaling, no collective in the data path);
-the value is the total over ranks divided by the slowest rank's device time.
+With N > 1 every rank runs its own independent request of the same shape (the path has no exchange
+step: weak scaling, no collective in the data path); the value is the total over ranks divided by the
+slowest rank's device time.  Started under torch.distributed.run the ranks come from the environment;
+started plainly with --gpus N > 1 the script starts the N ranks itself (one process per GPU,
+rendezvous on 127.0.0.1) and rank 0 prints the one JSON line.
 """
 from __future__ import annotations
 
@@ -98,7 +100,7 @@ def algorithmic_flops(profile, req):
 def oracle_sample_run(w, rows):
     """Runs the float64 checker on the packed rows `rows`; returns (seconds, visible pairs)."""
     import oracle
-    from tests.helpers import f64
+    from oracle.harness import f64
     p, lay = w.profile, w.layout
     rows = np.asarray(rows, dtype=np.int64)
     inv = oracle.inverse_row_map(w.prot_rows, lay.n_rows)
@@ -168,7 +170,7 @@ def run_reference(args, rank, world):
     sec = float(np.mean(times))
     tok_s = lay.n_rows / (sec * all_pairs / pairs)
     cores = os.cpu_count()
-    line = dict(metric="mla_online_prefill_tokens_per_s_per_layer", value=tok_s, unit="tokens/s", n_gpus=args.gpus,
+    line = dict(metric="mla_online_prefill_tokens_per_s_per_layer", value=tok_s, unit="tokens/s", n_gpus=world,
                 steps=args.steps, warmup=args.warmup, ms_per_step=sec * 1e3 * all_pairs / pairs,
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
                 impl="reference", config=dict(workload=name, T=lay.n_rows, n_prot=len(prot)),
@@ -313,7 +315,7 @@ def main():
     ap.add_argument("--regime", default="mandated", choices=["mandated", "sharp"])
     ap.add_argument("--oracle-pairs", type=int, default=150_000_000,
                     help="visible-pair budget of the CPU checker sample (about 10-30 s of host work)")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--protect-bp", type=int, default=None,
                     help="override the share of protected document rows (basis points), e.g. the paper's controller "
@@ -327,6 +329,9 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rk" else args.warmup
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started plainly: bring up one rank per GPU ourselves (the same launch torch.distributed.run does)
+        sys.exit(rkdist.spawn_ranks(args.gpus, [os.path.abspath(__file__)] + sys.argv[1:]))
     rank, world, local_rank = rkdist.env_ranks()
     if args.impl == "reference":
         run_reference(args, rank, world)
@@ -352,8 +357,6 @@ def main():
                                 device=dev, regime=args.regime)
         if ctx is None:
             ctx = rk.Context.from_profile(prof)
-            if os.environ.get("RK_DEBUG_FLAGS"):      # timing experiments only; results are meaningless then
-                ctx.rk_set_debug_flags(int(os.environ["RK_DEBUG_FLAGS"]))
         layers.append((wl, ctx.rk_request_create(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, prot)))
     w, req = layers[0]
     prof, lay = w.profile, w.layout
@@ -414,8 +417,10 @@ def main():
     clocks = sampler.summary()
 
     # end to end through the host-buffer entry point (H2D of the request inputs + D2H of y per step)
+    # measured at N = 1 only: every rank would pin its own copy of the inputs (about 10 GB at 256K), and the
+    # host-to-device copies of N ranks share the host's memory and PCIe paths, which this path does not model
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and world == 1:
         pin = lambda x: x.to("cpu").pin_memory()
         host = [(pin(wl.kv), pin(wl.q_g), pin(wl.q_l), pin(wl.z_off)) for wl, _ in layers]
         y_h = torch.empty((req.T, prof.d_model), dtype=torch.bfloat16).pin_memory()
@@ -507,7 +512,7 @@ def main():
         dt, pairs, out = oracle_sample_run(w, rows)
         allp = total_pairs(prof, req)          # layer 0 (the layers have the same layout, own protected rows)
         # while the sample is at hand: parity of this very run against the checker
-        from tests.helpers import rel_l2
+        from oracle.harness import rel_l2
         y_gpu = bufs["y"][torch.as_tensor(rows, device=dev)].float().cpu().numpy().astype(np.float64)
         cpu_baseline = dict(value=req.T / (dt * allp / pairs), unit="tokens/s (per layer)", cores=os.cpu_count(), kind="oracle",
                             threads=torch.get_num_threads(),

@@ -95,6 +95,19 @@ const char* rk_status_string(rk_status s);
 
 /* Creates a context on the CURRENT CUDA device.  Copies the profile (including global_heads). */
 rk_status rk_create(const rk_profile* profile, rk_ctx** out);
+/* Output-phase variant (Eq. offonline: z = W_a R^{-1}(O); Algorithm 2: RestorePhase(O_i, delta_i) per
+ * segment before SegmentedLSEMerge and R^{-1} in the z_online statement).  With RK_VALUE_PHASE the
+ * value of a key is its whole stored row [c | k_rope] (576 wide), not the latent alone, so an
+ * attention output carries 64 rotated dims.  Inside a segment they accumulate in the document's
+ * position-zero frame; RestorePhase turns them by R(+seg_delta[i]) into the request frame, where
+ * segments may be merged; R^{-1} turns row t's merged rope dims by R(-pos[t]), after which they
+ * depend on relative positions only.  The attention kernel does all three inside its running merge.
+ * What changes at the interface, and nothing else:
+ *   O_g / O_l (and O_part / O of rk_segmented_merge_phase) rows are 576 wide, rope dims last;
+ *   W_uv is [H][128][576];  rk_mla_off_build applies R^{-1} at the row's canonical position.
+ * The plain context (flags = 0) treats both maps as the identity: its values carry no rotated dims. */
+#define RK_VALUE_PHASE 1u
+rk_status rk_create_ex(const rk_profile* profile, uint32_t flags, rk_ctx** out);
 rk_status rk_destroy(rk_ctx* ctx);
 /* Message of the last failing call on this context (valid until the next call). */
 const char* rk_last_error(const rk_ctx* ctx);
@@ -102,12 +115,12 @@ const char* rk_last_error(const rk_ctx* ctx);
 rk_status rk_poll_status(rk_ctx* ctx, void* stream);
 /* Per-wait time limit of device-side waits, in milliseconds (default 2000). */
 rk_status rk_set_wait_limit_ms(rk_ctx* ctx, int32_t ms);
-/* Development switches of the attention kernel (0 = production).  Bit 0 removes the softmax
- * arithmetic and bit 2 the row-maximum exchange, for timing experiments (results are then
- * meaningless).  Bit 3 makes the load warp leave every ring stage empty, so the consumer's bounded
- * wait expires and the kernel returns with RK_ERR_TIMEOUT in the status word: the test of the
- * timeout path uses it together with a short rk_set_wait_limit_ms. */
-rk_status rk_set_debug_flags(rk_ctx* ctx, int32_t flags);
+/* Test hook for the timeout path (failure detection without a GPU fault): while `on` is non-zero the
+ * attention launches of this context use an instantiation whose load warp leaves every ring stage
+ * empty, so the consumers' bounded waits expire, the kernel drains and returns, and
+ * rk_poll_status() reports RK_ERR_TIMEOUT.  Results are not produced while it is on.  Use it
+ * together with a short rk_set_wait_limit_ms. */
+rk_status rk_test_starve_loads(rk_ctx* ctx, int32_t on);
 
 /* Request geometry object: validates the layout and the protected-row list (Eq. protected;
  * the list is data here), builds row positions, per-segment relocation tables
@@ -152,9 +165,23 @@ rk_status rk_mla_online_attn(rk_ctx* ctx, const rk_request* req, const void* kv,
  *   O_part   device [n_parts][n_rows][n_heads][512], bf16 (part_dtype 0) or fp32 (part_dtype 1)
  *   lse_part device fp32 [n_parts][n_rows][n_heads]; -inf marks an empty part (its O is ignored)
  *   O device bf16 [n_rows][n_heads][512], lse device fp32 [n_rows][n_heads]
- * All parts empty gives O = 0, lse = -inf. */
+ * All parts empty gives O = 0, lse = -inf.  n_parts <= 4096. */
 rk_status rk_segmented_merge(rk_ctx* ctx, int32_t n_parts, int64_t n_rows, int32_t n_heads, const void* O_part,
                              int32_t part_dtype, const float* lse_part, void* O, float* lse, void* stream);
+
+/* The same merge for per-segment partial results of the output-phase variant (Algorithm 2:
+ * RestorePhase, then SegmentedLSEMerge, then R^{-1}).  Part j is the partial result against the
+ * canonical rows of segment seg_begin + j: its 64 rope dims (the last of 576) are in that document's
+ * frame and are turned by R(+seg_delta[seg_begin + j]) before they are added.
+ *   O_part   device [n_parts][n_rows][n_heads][576], bf16 (part_dtype 0) or fp32 (part_dtype 1)
+ *   lse_part device fp32 [n_parts][n_rows][n_heads]; -inf marks an empty part (its O is ignored)
+ *   row_pos  device int32 [n_rows]: request position of each row, whose merged rope dims are turned by
+ *            R(-row_pos[r]); NULL leaves the result in the request frame
+ *   O device bf16 [n_rows][n_heads][576], lse device fp32 [n_rows][n_heads]
+ * seg_begin + n_parts <= number of segments of `req`; n_parts <= 4096. */
+rk_status rk_segmented_merge_phase(rk_ctx* ctx, const rk_request* req, int32_t seg_begin, int32_t n_parts, int64_t n_rows,
+                                   int32_t n_heads, const void* O_part, int32_t part_dtype, const float* lse_part,
+                                   const int32_t* row_pos, void* O, float* lse, void* stream);
 
 /* (4) Group-aligned sliced first output projection (Eq. offonline; Algorithm 2: z_online):
  * per head o = W_uv[h] O_lat (512 -> 128), then the head's 128-column slice of its group's W_a:
@@ -177,8 +204,10 @@ rk_status rk_group_sliced_proj(rk_ctx* ctx, const rk_request* req, const void* O
  * holds that array until the process exits.  The call allocates and frees nothing.
  *  - Requests whose scratch need (rk_workspace_bytes) exceeds 32 MiB are rejected with
  *    RK_ERR_WORKSPACE and a message; use rk_group_sliced_proj with your own workspace then.
- *  - The first call on each device looks up the array's device address (the context's device
- *    must be current); make that first call before starting any stream capture.
+ *  - rk_create looks up the array's device address on the context's device (the lookup makes the
+ *    runtime place the array on that device, which may allocate and synchronise once); the entry
+ *    point itself only reads the cached address, so create the context before any stream capture.
+ *    The context's device must be current when the entry point is called.
  *  - All calls, from all contexts and streams of a process, share the one array, and it keeps
  *    whatever the previous call left in it.  Nothing in it needs to start at zero.  Two calls
  *    whose kernels overlap on the GPU (different streams) race on it: serialise them.
@@ -187,7 +216,8 @@ rk_status rk_group_sliced_proj_static(rk_ctx* ctx, const rk_request* req, const 
                                       const void* W_uv, const void* W_a, void* z_on_g, void* z_on_l, void* stream);
 
 /* (5) Add the offline MLA-Off artifact and run the shared second projection (Algorithm 2:
- * RestoreAndReplace, then W_b z; "replaced, never double counted"):
+ * RestoreAndReplace, then W_b z; the paragraph after Eq. protected: a row in A takes the online Local
+ * value in place of the artifact's, the two are never added):
  *   z[t] = z_on_g[t] + (t in A ? z_on_l[slot(t)] : z_off[t]);  y = W_b z.
  *   z_off device bf16 [n_off_rows][G*r_o] (packed rows; rows in A are never read)
  *   W_b   device bf16 [d_model][G*r_o], may be NULL to stop at z
@@ -270,7 +300,11 @@ typedef struct rk_layer_buffers {
   size_t workspace_bytes;
 } rk_layer_buffers;
 
-/* One whole layer from HOST inputs: copies kv, q_g, q_l, z_off host->device (use pinned host
+/* rk_layer_host and rk_layer_stack_host use one set of internal copy streams and events per
+ * context: at most one of them may be running on a context at any time (two host threads must not
+ * call them concurrently on the same rk_ctx; use one context per thread).
+ *
+ * One whole layer from HOST inputs: copies kv, q_g, q_l, z_off host->device (use pinned host
  * memory; pageable memory works but serialises), runs (2), (4), (5), copies y device->host and
  * synchronises `stream`.  Weights stay resident on the device.  Copies that the running kernel
  * does not need yet travel on an internal second stream beside it (the Local pass needs only kv

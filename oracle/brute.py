@@ -4,7 +4,8 @@ transposed operand in either shows up as a disagreement.  Only for a few tokens.
 
 Test infrastructure; cites the same passages: Eq. rope (key re-rotation), Algorithm 2
 (Global heads on every row, Local heads on protected rows), Eq. offonline / factorization
-(sliced W_a, shared W_b), "replaced, never double counted".
+(sliced W_a, shared W_b), RestoreAndReplace (a protected row takes the online Local value in place of
+the artifact; the two are never added).
 """
 from __future__ import annotations
 

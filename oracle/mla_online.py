@@ -217,7 +217,8 @@ def mla_online_rows(rows: np.ndarray, q_g_rows: np.ndarray, q_l_rows, kv: np.nda
     q_g_rows [n, G, d_qk]: Global-head queries of those rows.
     q_l_rows: dict {packed row -> [L, d_qk]} (or array aligned with the protected ones among
     `rows`, in the order they appear) with the Local-head queries of the protected rows.
-    Steps (Algorithm 2 after the merge; Eq. offonline; "replaced, never double counted"):
+    Steps (Algorithm 2 after the merge; Eq. offonline; RestoreAndReplace: a protected row takes the
+    online Local value in place of the artifact, the two are never added):
       O_G   = attention of the Global heads, every row
       O_L,A = attention of the Local heads, protected rows only
       z_on_g[t, g] = contribution of group g's Global head

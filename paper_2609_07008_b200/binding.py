@@ -54,7 +54,7 @@ class rk_layer_io(C.Structure):
 
 
 EXPORTS = ["rk_version", "rk_status_string", "rk_create", "rk_destroy", "rk_last_error", "rk_poll_status",
-           "rk_set_wait_limit_ms", "rk_set_debug_flags", "rk_request_create", "rk_request_destroy", "rk_check_request",
+           "rk_set_wait_limit_ms", "rk_test_starve_loads", "rk_request_create", "rk_request_destroy", "rk_check_request",
            "rk_request_get_info", "rk_workspace_bytes", "rk_relocate_q", "rk_mla_online_attn",
            "rk_segmented_merge", "rk_group_sliced_proj", "rk_group_sliced_proj_static", "rk_combine_offline",
            "rk_layer_host", "rk_layer_stack_host", "rk_mla_off_workspace_bytes", "rk_mla_off_build",
@@ -77,7 +77,7 @@ def _load() -> C.CDLL:
     lib.rk_destroy.argtypes = [vp]
     lib.rk_poll_status.argtypes = [vp, vp]
     lib.rk_set_wait_limit_ms.argtypes = [vp, i32]
-    lib.rk_set_debug_flags.argtypes = [vp, i32]
+    lib.rk_test_starve_loads.argtypes = [vp, i32]
     lib.rk_request_create.argtypes = [vp, C.POINTER(rk_layout), C.POINTER(i32), i64, C.POINTER(vp)]
     lib.rk_request_destroy.argtypes = [vp]
     lib.rk_check_request.argtypes = [C.POINTER(rk_layout), C.POINTER(i32), i64, C.c_char_p, C.c_size_t]
@@ -119,6 +119,12 @@ def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
         return None
     assert t.is_contiguous(), "tensors passed to the library must be contiguous"
     return t.data_ptr()
+
+
+def _empty(shape, dtype, device):
+    """Every buffer the binding allocates on behalf of the caller (outputs, scratch) comes from here, so a
+    caller with its own memory pool -- or a test that wants guard zones around the outputs -- can replace it."""
+    return torch.empty(shape, dtype=dtype, device=device)
 
 
 def _stream() -> int:
@@ -184,8 +190,8 @@ class Context:
     def rk_set_wait_limit_ms(self, ms: int):
         self.check(lib.rk_set_wait_limit_ms(self.handle, ms))
 
-    def rk_set_debug_flags(self, flags: int):
-        self.check(lib.rk_set_debug_flags(self.handle, flags))
+    def rk_test_starve_loads(self, on: bool):
+        self.check(lib.rk_test_starve_loads(self.handle, 1 if on else 0))
 
     def rk_request_create(self, seg_off, seg_delta, seg_has_artifact, prot_rows) -> "Request":
         return Request(self, seg_off, seg_delta, seg_has_artifact, prot_rows)
@@ -197,7 +203,7 @@ class Context:
         n_rows, n_heads, w = q_rope_view.shape
         assert w == 64 and q_rope_view.stride(2) == 1 and q_rope_view.dtype == torch.bfloat16
         if out is None:
-            out = torch.empty((seg_end - seg_begin, n_rows, n_heads, 64), dtype=torch.bfloat16,
+            out = _empty((seg_end - seg_begin, n_rows, n_heads, 64), dtype=torch.bfloat16,
                               device=q_rope_view.device)
         self.check(lib.rk_relocate_q(self.handle, req.handle, q_rope_view.data_ptr(), n_rows, n_heads,
                                      q_rope_view.stride(0), q_rope_view.stride(1), seg_begin, seg_end,
@@ -207,11 +213,11 @@ class Context:
     def rk_mla_online_attn(self, req, kv, q_g, q_l, O_g=None, lse_g=None, O_l=None, lse_l=None):
         dev = kv.device
         if q_g is not None and O_g is None:
-            O_g = torch.empty((req.T, self.n_groups, 512), dtype=torch.bfloat16, device=dev)
-            lse_g = torch.empty((req.T, self.n_groups), dtype=torch.float32, device=dev)
+            O_g = _empty((req.T, self.n_groups, 512), dtype=torch.bfloat16, device=dev)
+            lse_g = _empty((req.T, self.n_groups), dtype=torch.float32, device=dev)
         if q_l is not None and O_l is None:
-            O_l = torch.empty((req.A, self.n_local, 512), dtype=torch.bfloat16, device=dev)
-            lse_l = torch.empty((req.A, self.n_local), dtype=torch.float32, device=dev)
+            O_l = _empty((req.A, self.n_local, 512), dtype=torch.bfloat16, device=dev)
+            lse_l = _empty((req.A, self.n_local), dtype=torch.float32, device=dev)
         self.check(lib.rk_mla_online_attn(self.handle, req.handle, _ptr(kv), _ptr(q_g), _ptr(q_l), _ptr(O_g),
                                           _ptr(lse_g), _ptr(O_l), _ptr(lse_l), _stream()))
         return O_g, lse_g, O_l, lse_l
@@ -221,8 +227,8 @@ class Context:
         assert d == 512 and lse_part.shape == (P, n_rows, n_heads) and lse_part.dtype == torch.float32
         dt = {torch.bfloat16: 0, torch.float32: 1}[O_part.dtype]
         if O is None:
-            O = torch.empty((n_rows, n_heads, 512), dtype=torch.bfloat16, device=O_part.device)
-            lse = torch.empty((n_rows, n_heads), dtype=torch.float32, device=O_part.device)
+            O = _empty((n_rows, n_heads, 512), dtype=torch.bfloat16, device=O_part.device)
+            lse = _empty((n_rows, n_heads), dtype=torch.float32, device=O_part.device)
         self.check(lib.rk_segmented_merge(self.handle, P, n_rows, n_heads, _ptr(O_part), dt, _ptr(lse_part),
                                           _ptr(O), _ptr(lse), _stream()))
         return O, lse
@@ -231,11 +237,11 @@ class Context:
         dev = W_uv.device
         width = self.n_groups * self.o_rank
         if O_g is not None and z_on_g is None:
-            z_on_g = torch.empty((req.T, width), dtype=torch.bfloat16, device=dev)
+            z_on_g = _empty((req.T, width), dtype=torch.bfloat16, device=dev)
         if O_l is not None and z_on_l is None:
-            z_on_l = torch.empty((req.A, width), dtype=torch.bfloat16, device=dev)
+            z_on_l = _empty((req.A, width), dtype=torch.bfloat16, device=dev)
         if workspace is None:
-            workspace = torch.empty(max(req.workspace_bytes, 256), dtype=torch.uint8, device=dev)
+            workspace = _empty(max(req.workspace_bytes, 256), dtype=torch.uint8, device=dev)
         self.check(lib.rk_group_sliced_proj(self.handle, req.handle, _ptr(O_g), _ptr(O_l), _ptr(W_uv), _ptr(W_a),
                                             _ptr(z_on_g), _ptr(z_on_l), _ptr(workspace), workspace.numel(),
                                             _stream()))
@@ -261,9 +267,9 @@ class Context:
             s = lib.rk_protected_rows_workspace_bytes(T, S, C.byref(need))
             if s != 0:
                 raise RKError(s, "rk_protected_rows_workspace_bytes")
-            workspace = torch.empty(need.value, dtype=torch.uint8, device=device)
+            workspace = _empty(need.value, dtype=torch.uint8, device=device)
         if out is None:
-            out = (torch.empty(T, dtype=torch.int32, device=device), torch.empty(1, dtype=torch.int64, device=device))
+            out = (_empty(T, dtype=torch.int32, device=device), _empty(1, dtype=torch.int64, device=device))
         n_dirty = 0 if dirty_rows is None else dirty_rows.numel()
         self.check(lib.rk_protected_rows(self.handle, C.byref(lay), C.byref(pol), _ptr(dirty_rows), n_dirty, _ptr(scores),
                                          _ptr(out[0]), _ptr(out[1]), _ptr(workspace), workspace.numel(), _stream()))
@@ -279,8 +285,8 @@ class Context:
         assert p.dtype == torch.float32 and p.dim() == 2 and p.shape[1] == 6 and p.is_contiguous()
         n = p.shape[0]
         if k_out is None:
-            k_out = torch.empty(n, dtype=torch.uint8, device=p.device)
-            keep_out = torch.empty(n, dtype=torch.uint8, device=p.device)
+            k_out = _empty(n, dtype=torch.uint8, device=p.device)
+            keep_out = _empty(n, dtype=torch.uint8, device=p.device)
         self.check(lib.rk_moe_fanout(self.handle, _ptr(p), n, float(tau), int(bool(fence)), _ptr(k_out), _ptr(keep_out),
                                      _stream()))
         return k_out, keep_out
@@ -288,9 +294,9 @@ class Context:
     def rk_combine_offline(self, req, z_on_g, z_on_l, z_off, W_b, z=None, y=None):
         dev = z_on_g.device
         if z is None:
-            z = torch.empty((req.T, self.n_groups * self.o_rank), dtype=torch.bfloat16, device=dev)
+            z = _empty((req.T, self.n_groups * self.o_rank), dtype=torch.bfloat16, device=dev)
         if W_b is not None and y is None:
-            y = torch.empty((req.T, self.d_model), dtype=torch.bfloat16, device=dev)
+            y = _empty((req.T, self.d_model), dtype=torch.bfloat16, device=dev)
         self.check(lib.rk_combine_offline(self.handle, req.handle, _ptr(z_on_g), _ptr(z_on_l), _ptr(z_off),
                                           _ptr(W_b), _ptr(z), _ptr(y), _stream()))
         return z, y
@@ -299,11 +305,11 @@ class Context:
         """Offline artifact rows [row_begin, row_end): documents alone at position zero, Local heads."""
         n = row_end - row_begin
         if z_off_rows is None:
-            z_off_rows = torch.empty((n, self.n_groups * self.o_rank), dtype=torch.bfloat16, device=kv.device)
+            z_off_rows = _empty((n, self.n_groups * self.o_rank), dtype=torch.bfloat16, device=kv.device)
         ws = C.c_size_t()
         self.check(lib.rk_mla_off_workspace_bytes(req.handle, n, C.byref(ws)))
         if workspace is None:
-            workspace = torch.empty(max(ws.value, 256), dtype=torch.uint8, device=kv.device)
+            workspace = _empty(max(ws.value, 256), dtype=torch.uint8, device=kv.device)
         self.check(lib.rk_mla_off_build(self.handle, req.handle, _ptr(kv), row_begin, row_end, _ptr(q_l_rows),
                                         _ptr(W_uv), _ptr(W_a), _ptr(z_off_rows), _ptr(workspace), workspace.numel(),
                                         _stream()))
@@ -313,12 +319,12 @@ class Context:
         G, L, T, A = self.n_groups, self.n_local, req.T, req.A
         width = G * self.o_rank
         bf, f32 = torch.bfloat16, torch.float32
-        e = lambda shape, dt=bf: torch.empty(shape, dtype=dt, device=device)
+        e = lambda shape, dt=bf: _empty(shape, dtype=dt, device=device)
         return dict(kv=e((T, 576)), q_g=e((T, G, 576)), q_l=e((max(A, 1), L, 576)),
                     z_off=e((max(req.n_off_rows, 1), width)), O_g=e((T, G, 512)), O_l=e((max(A, 1), L, 512)),
                     z_on_g=e((T, width)), z_on_l=e((max(A, 1), width)), z=e((T, width)), y=e((T, self.d_model)),
                     lse_g=e((T, G), f32), lse_l=e((max(A, 1), L), f32),
-                    workspace=torch.empty(max(req.workspace_bytes, 256), dtype=torch.uint8, device=device))
+                    workspace=_empty(max(req.workspace_bytes, 256), dtype=torch.uint8, device=device))
 
     def rk_layer_host(self, req, kv_h, q_g_h, q_l_h, z_off_h, W_uv, W_a, W_b, bufs: dict, y_h: torch.Tensor):
         """Whole layer from pinned host tensors: H2D copies, the three device calls, D2H of y, sync."""

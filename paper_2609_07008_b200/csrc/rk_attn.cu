@@ -30,54 +30,52 @@
 #include "rk_internal.h"
 
 namespace rk {
-#ifdef RK_TRACE
-__device__ long long g_trace[4 * 16384];
-// records (tag, clock64) pairs of CTA 0; the events of the first ((debug >> 8) << 6) key tiles are skipped
-// so that a window late in a long launch can be looked at
-#define RK_TR(role, tag) do { if (blockIdx.x == 0 && lane == 0) { if (tr_skip[role] > 0) --tr_skip[role]; else if (tr_n[role] < 8190) { g_trace[(role) * 16384 + 2 * tr_n[role]] = (tag); g_trace[(role) * 16384 + 2 * tr_n[role] + 1] = clock64(); ++tr_n[role]; } } } while (0)
-// cheap wait-time accumulators (clock deltas summed in registers, written once at the end of CTA 0)
-#define RK_ACC_T0() const long long acc_t0 = clock64()
-#define RK_ACC(i) do { acc[i] += clock64() - acc_t0; } while (0)
-#define RK_ACC_DUMP(role, n) do { if (blockIdx.x == 0 && lane == 0) for (int i_ = 0; i_ < (n); ++i_) g_trace[3 * 16384 + 32 * (role) + i_] = acc[i_]; } while (0)
-#else
-#define RK_TR(role, tag) do { } while (0)
-#define RK_ACC_T0() do { } while (0)
-#define RK_ACC(i) do { } while (0)
-#define RK_ACC_DUMP(role, n) do { } while (0)
-#endif
 namespace {
 
 constexpr int kAttnThreads = 384;       // 4 role warps + 8 softmax warps
-constexpr int kStages = 4;                // ring of 32 KB stages (two 16 KB TMA boxes each)
 constexpr uint32_t kChunkBytes = 16384;  // 128 keys x 64 dims bf16
 constexpr uint32_t kStageBytes = 2 * kChunkBytes;
 constexpr uint32_t kQChunkBytes = 8192;  // 64 rows x 64 dims bf16
 
-// shared memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t kOffQLat = 0;                                // latent dims 0-255: 4 chunks (dims 256-511 live in TMEM)
-constexpr uint32_t kOffQPristine = kOffQLat + 4 * kQChunkBytes;  // rope chunk as loaded
-constexpr uint32_t kOffQRot = kOffQPristine + kQChunkBytes;      // 2 rotated rope chunks
-constexpr uint32_t kOffP = kOffQRot + 2 * kQChunkBytes;          // 4 sub-chunks [64 x 64 keys]
-constexpr uint32_t kOffRing = kOffP + 4 * kQChunkBytes;
-constexpr uint32_t kOffBars = kOffRing + kStages * kStageBytes;
-// barrier indices (8 bytes each)
-constexpr int kBarQFull = 0, kBarQFree = 1, kBarQrReady = 2 /*2*/, kBarQrFree = 4 /*2*/, kBarRingFull = 6,
-              kBarRingEmpty = kBarRingFull + kStages, kBarSFull = kBarRingEmpty + kStages,
-              kBarSFree = kBarSFull + 1, kBarPReady = kBarSFree + 1, kBarPvDone = kBarPReady + 1,
-              kBarQhFull = kBarPvDone + 1, kBarQhDone = kBarQhFull + 1, kNumBars = kBarQhDone + 1;
-constexpr uint32_t kOffTmemPtr = kOffBars + kNumBars * 8;
-constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
-constexpr uint32_t kOffXchg = kOffAbort + 8;                 // u64 [2 parity][4 parts][64]: (seq << 32) | value
-constexpr uint32_t kSmemUsed = kOffXchg + 2 * 4 * 64 * 8;
-constexpr uint32_t kSmemBytes = kSmemUsed + 1024;            // + alignment slack
+// Two instantiations share this file.  The plain one (values = the 512-wide latent) keeps latent dims
+// 256-511 of the Q tile in tensor memory and runs a four-stage ring.  The output-phase one (values = the
+// whole stored row, latent and rope dims; Eq. offonline's inverse output RoPE, Algorithm 2's RestorePhase)
+// needs 32 more accumulator columns for the rope part of O, which do not fit beside the tensor-memory Q
+// half (256 + 128 + 128 + 32 > 512): it keeps all of Q in shared memory and runs a three-stage ring.
+template <bool kPhase>
+struct Cfg {
+  static constexpr int kStages = kPhase ? 3 : 4;          // ring of 32 KB stages (two 16 KB TMA boxes each)
+  static constexpr int kQSmemChunks = kPhase ? 8 : 4;     // 64-dim latent chunks of Q kept in shared memory
+  static constexpr int kStagesPerKeyTile = kPhase ? 10 : 9;  // K: 5, V: 4, rope part of V: 1
+  static constexpr int kOW = kPhase ? kDQK : kDLatent;    // width of an output row
+  // shared memory map (offsets from a 1024-byte aligned base)
+  static constexpr uint32_t kOffQLat = 0;
+  static constexpr uint32_t kOffQPristine = kOffQLat + kQSmemChunks * kQChunkBytes;  // rope chunk as loaded
+  static constexpr uint32_t kOffQRot = kOffQPristine + kQChunkBytes;                 // 2 rotated rope chunks
+  static constexpr uint32_t kOffP = kOffQRot + 2 * kQChunkBytes;                     // 4 sub-chunks [64 x 64 keys]
+  static constexpr uint32_t kOffRing = kOffP + 4 * kQChunkBytes;
+  static constexpr uint32_t kOffBars = kOffRing + kStages * kStageBytes;
+  // barrier indices (8 bytes each)
+  static constexpr int kBarQFull = 0, kBarQFree = 1, kBarQrReady = 2 /*2*/, kBarQrFree = 4 /*2*/, kBarRingFull = 6,
+                       kBarRingEmpty = kBarRingFull + kStages, kBarSFull = kBarRingEmpty + kStages,
+                       kBarSFree = kBarSFull + 1, kBarPReady = kBarSFree + 1, kBarPvDone = kBarPReady + 1,
+                       kBarQhFull = kBarPvDone + 1, kBarQhDone = kBarQhFull + 1, kNumBars = kBarQhDone + 1;
+  static constexpr uint32_t kOffTmemPtr = kOffBars + kNumBars * 8;
+  static constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
+  static constexpr uint32_t kOffXchg = kOffAbort + 8;         // u64 [2 parity][4 parts][64]: (seq << 32) | value
+  static constexpr uint32_t kSmemUsed = kOffXchg + 2 * 4 * 64 * 8;
+  static constexpr uint32_t kSmemBytes = kSmemUsed + 1024;    // + alignment slack
+};
 
 // TMEM columns
-constexpr uint32_t kColO = 0;    // two halves of 128 columns
-constexpr uint32_t kColS = 256;  // one 128-column score buffer
-constexpr uint32_t kColQ = 384;  // latent dims 256-511 of the Q tile as a TMEM A operand (both lane halves hold the rows)
+constexpr uint32_t kColO = 0;     // two halves of 128 columns
+constexpr uint32_t kColS = 256;   // one 128-column score buffer
+constexpr uint32_t kColQ = 384;   // plain: latent dims 256-511 of the Q tile as a TMEM A operand (both lane halves hold the rows)
+constexpr uint32_t kColOr = 384;  // output-phase: the 64 rope dims of O (N = 64 folds onto 32 columns)
 
 constexpr uint32_t kIdescQK = umma_idesc_bf16(128, 256, 0, 0);
 constexpr uint32_t kIdescPV = umma_idesc_bf16(128, 256, 0, 1);
+constexpr uint32_t kIdescPVr = umma_idesc_bf16(128, 64, 0, 1);  // rope part of the value: 32 dims per CTA
 
 // wait tags reported on timeout
 enum { W_QFULL = 1, W_QFREE, W_QRREADY, W_QRFREE, W_RINGFULL, W_RINGEMPTY, W_SFULL, W_PREADY, W_PVDONE, W_DRAIN, W_SFREE, W_QHFULL, W_QHDONE };
@@ -138,6 +136,7 @@ __device__ __forceinline__ AttnWorkItem get_work(const AttnParams& p, int w) {
 // sequence.  A stage holds two 16 KB boxes: two 64-dim K chunks (QK^T), the single rope chunk,
 // or the two 64-dim halves of this CTA's 128 output dims (PV; 16 KB apart = the descriptor's
 // leading byte offset).
+template <int kStages>
 struct RingPos {
   uint32_t it = 0;  // stages used so far
   __device__ uint32_t stage() const { return it % kStages; }
@@ -192,6 +191,15 @@ __device__ __forceinline__ bool quad_exchange(volatile unsigned long long* xbuf,
 #define quad_exchange_max quad_exchange<true>
 #define quad_exchange_sum quad_exchange<false>
 
+// (cos, sin) of d * theta_j for an integer position difference d (any sign, up to 2^30): the angle is
+// reduced in double precision in units of turns (theta_j / 2 pi is a host-computed double), so that the
+// float sincospi sees an argument in [-1, 1] whatever the size of d
+__device__ __forceinline__ void rope_cs(const AttnParams& p, int d, int j, float& c, float& s) {
+  const double t = (double)d * p.rope_turns[j];
+  const float f = (float)(t - rint(t));
+  sincospif(2.f * f, &s, &c);
+}
+
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -200,8 +208,15 @@ __device__ __forceinline__ float fast_exp2(float x) {
 
 }  // namespace
 
+// kStarve: test instantiation whose load warp leaves every ring stage empty, so that the consumers'
+// bounded waits expire and the kernel returns with RK_ERR_TIMEOUT in the status word (the test of the
+// timeout path launches it; the production instantiation carries no such switch in its loops).
+// kPhase: the output-phase instantiation (see Cfg).
+template <bool kPhase, bool kStarve>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     rk_mla_attn_kernel(const __grid_constant__ AttnParams p) {
+  using C = Cfg<kPhase>;
+  constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -211,43 +226,35 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
   const int pair = blockIdx.x >> 1;
   const bool leader = (crank == 0);
 
-  auto bar = [&](int i) -> uint32_t { return smem_base + kOffBars + 8u * i; };
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffAbort);
-  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + kOffTmemPtr);
+  auto bar = [&](int i) -> uint32_t { return smem_base + C::kOffBars + 8u * i; };
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + C::kOffAbort);
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + C::kOffTmemPtr);
   const uint64_t limit = p.wait_ns;
-#ifdef RK_TRACE
-  int tr_n[4] = {0, 0, 0, 0};
-  const int tr_tiles = (p.debug >> 8) << 6;  // events per key tile: issuer 23, softmax 5, producer 9
-  int tr_skip[4] = {23 * tr_tiles, 5 * tr_tiles, 9 * tr_tiles, 0};
-  if (p.debug & 16) tr_skip[0] = tr_skip[1] = tr_skip[2] = 0x7fffffff;  // accumulators only, no event records
-  long long acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-  const long long acc_start = clock64();
-#endif
 
-  for (int i = threadIdx.x; i < 512; i += kAttnThreads) reinterpret_cast<volatile unsigned long long*>(smem + kOffXchg)[i] = 0ull;
+  for (int i = threadIdx.x; i < 512; i += kAttnThreads) reinterpret_cast<volatile unsigned long long*>(smem + C::kOffXchg)[i] = 0ull;
   if (threadIdx.x == 0) {
     *abort_flag = 0;
-    mbar_init(bar(kBarQFull), 1);
-    mbar_init(bar(kBarQFree), 1);
+    mbar_init(bar(C::kBarQFull), 1);
+    mbar_init(bar(C::kBarQFree), 1);
     for (int b = 0; b < 2; ++b) {
-      mbar_init(bar(kBarQrReady + b), 2);
-      mbar_init(bar(kBarQrFree + b), 1);
+      mbar_init(bar(C::kBarQrReady + b), 2);
+      mbar_init(bar(C::kBarQrFree + b), 1);
     }
-    mbar_init(bar(kBarSFull), 1);
-    mbar_init(bar(kBarSFree), 16);   // every softmax warp of the pair has read the score buffer
-    mbar_init(bar(kBarQhFull), 1);   // this CTA's upper Q half has landed in its ring stage
-    mbar_init(bar(kBarQhDone), 16);  // every softmax warp of the pair has moved its part into TMEM
+    mbar_init(bar(C::kBarSFull), 1);
+    mbar_init(bar(C::kBarSFree), 16);   // every softmax warp of the pair has read the score buffer
+    mbar_init(bar(C::kBarQhFull), 1);   // this CTA's upper Q half has landed in its ring stage
+    mbar_init(bar(C::kBarQhDone), 16);  // every softmax warp of the pair has moved its part into TMEM
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar(kBarRingFull + s), 1);
-      mbar_init(bar(kBarRingEmpty + s), 1);
+      mbar_init(bar(C::kBarRingFull + s), 1);
+      mbar_init(bar(C::kBarRingEmpty + s), 1);
     }
-    mbar_init(bar(kBarPReady), 16);
-    mbar_init(bar(kBarPvDone), 1);
+    mbar_init(bar(C::kBarPReady), 16);
+    mbar_init(bar(C::kBarPvDone), 1);
     fence_mbar_init_cluster();
   }
   if (warp == 0) {
     __syncwarp();
-    tmem_alloc<2>(smem_base + kOffTmemPtr, 512);
+    tmem_alloc<2>(smem_base + C::kOffTmemPtr, 512);
     tmem_relinquish<2>();
   }
   tc_fence_before_sync();
@@ -264,7 +271,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       tma_prefetch_desc(&p.tm_q);
       tma_prefetch_desc(&p.tm_kv);
     }
-    RingPos rp;
+    RingPos<kStages> rp;
     uint32_t qfree_phase = 0;
     bool ok = true;
     int n_done = 0;
@@ -273,25 +280,45 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     auto fill = [&](int col0, int col1, int row, int w) -> bool {
       const uint32_t s = rp.stage();
       if (rp.it >= (uint32_t)kStages) {
-        RK_ACC_T0();
-        if (!mbar_wait_bounded<false>(bar(kBarRingEmpty + s), rp.parity() ^ 1u, limit, abort_flag, p.status,
+        if (!mbar_wait_bounded<false>(bar(C::kBarRingEmpty + s), rp.parity() ^ 1u, limit, abort_flag, p.status,
                                       W_RINGEMPTY, w))
           return false;
-        RK_ACC(0);
       }
-      if (p.debug & 8) {  // test switch: leave the stage empty so that the consumer's bounded wait expires
+      if constexpr (kStarve) {  // leave the stage empty: the consumer's bounded wait expires
         rp.advance();
         return true;
       }
-      RK_TR(2, 1);
       if (elect_one()) {
-        const uint32_t full_local = bar(kBarRingFull + s);
+        const uint32_t full_local = bar(C::kBarRingFull + s);
         const uint32_t nbox = (col1 >= 0) ? 2u : 1u;
         if (leader) mbar_arrive_expect_tx(full_local, 2 * nbox * kChunkBytes);
         const uint32_t full_remote = mapa_shared(full_local, 0);
-        const uint32_t dst = smem_base + kOffRing + s * kStageBytes;
+        const uint32_t dst = smem_base + C::kOffRing + s * kStageBytes;
         tma_load_2d_pair_hint(dst, &p.tm_kv, full_remote, col0, row, pol_kv);
         if (col1 >= 0) tma_load_2d_pair_hint(dst + kChunkBytes, &p.tm_kv, full_remote, col1, row, pol_kv);
+      }
+      __syncwarp();
+      rp.advance();
+      return true;
+    };
+    auto fill2 = [&](int col, int row_a, int row_b, int w) -> bool {  // one stage: the same columns of two row blocks
+      const uint32_t s = rp.stage();
+      if (rp.it >= (uint32_t)kStages) {
+        if (!mbar_wait_bounded<false>(bar(C::kBarRingEmpty + s), rp.parity() ^ 1u, limit, abort_flag, p.status,
+                                      W_RINGEMPTY, w))
+          return false;
+      }
+      if constexpr (kStarve) {
+        rp.advance();
+        return true;
+      }
+      if (elect_one()) {
+        const uint32_t full_local = bar(C::kBarRingFull + s);
+        if (leader) mbar_arrive_expect_tx(full_local, 4 * kChunkBytes);
+        const uint32_t full_remote = mapa_shared(full_local, 0);
+        const uint32_t dst = smem_base + C::kOffRing + s * kStageBytes;
+        tma_load_2d_pair_hint(dst, &p.tm_kv, full_remote, col, row_a, pol_kv);
+        tma_load_2d_pair_hint(dst + kChunkBytes, &p.tm_kv, full_remote, col, row_b, pol_kv);
       }
       __syncwarp();
       rp.advance();
@@ -309,39 +336,47 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           const int col = 256 * h + 128 * (int)crank;
           if (!fill(col, col + 64, seg_row0 + kb + kh * 128, w)) return false;
         }
+      if constexpr (kPhase) {
+        // rope part of the value: this CTA's 32 of the 64 rope dims for all 256 keys of the tile.  The box is
+        // the usual 64 columns wide and starts at this CTA's first dim (544 for the second CTA: the columns
+        // beyond the row's 576 are zero-filled and never read), so both CTAs find their dims at the same
+        // shared-memory offset, which the single MMA descriptor of the pair requires.
+        const int col = kDLatent + 32 * (int)crank;
+        if (!fill2(col, seg_row0 + kb, seg_row0 + kb + 128, w)) return false;
+      }
       return true;
     };
     for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs, ++n_done) {
       const AttnWorkItem item = get_work(p, w);
       // Q tile: wait until the previous tile's QK^T MMAs have finished reading it
       if (n_done > 0) {
-        ok = mbar_wait_bounded<false>(bar(kBarQFree), qfree_phase, limit, abort_flag, p.status, W_QFREE, w);
+        ok = mbar_wait_bounded<false>(bar(C::kBarQFree), qfree_phase, limit, abort_flag, p.status, W_QFREE, w);
         qfree_phase ^= 1;
         if (!ok) break;
       }
       const int qrow = item.tile * kAttnRowsPerPair + (int)crank * kAttnRowsPerCta;
-      if (elect_one()) {  // lower latent half and the rope chunk stay in shared memory for the whole row tile
-        mbar_arrive_expect_tx(bar(kBarQFull), 5 * kQChunkBytes);
-        for (int d = 0; d < 4; ++d)
-          tma_load_2d_hint(smem_base + kOffQLat + d * kQChunkBytes, &p.tm_q, bar(kBarQFull), d * 64, qrow, pol_q);
-        tma_load_2d_hint(smem_base + kOffQPristine, &p.tm_q, bar(kBarQFull), kDLatent, qrow, pol_q);
+      if (elect_one()) {  // latent chunks kept in shared memory and the rope chunk stay for the whole row tile
+        mbar_arrive_expect_tx(bar(C::kBarQFull), (C::kQSmemChunks + 1) * kQChunkBytes);
+        for (int d = 0; d < C::kQSmemChunks; ++d)
+          tma_load_2d_hint(smem_base + C::kOffQLat + d * kQChunkBytes, &p.tm_q, bar(C::kBarQFull), d * 64, qrow, pol_q);
+        tma_load_2d_hint(smem_base + C::kOffQPristine, &p.tm_q, bar(C::kBarQFull), kDLatent, qrow, pol_q);
       }
       __syncwarp();
       // Upper latent half (dims 256-511): staged through one ring stage, from where the softmax warps move
       // it into tensor memory.  Each CTA loads its own rows and signals its own barrier; the issuer lets go
       // of the ring position once both CTAs have finished the move.
-      {
+      if constexpr (!kPhase) {
         const uint32_t s = rp.stage();
         if (rp.it >= (uint32_t)kStages) {
-          ok = mbar_wait_bounded<false>(bar(kBarRingEmpty + s), rp.parity() ^ 1u, limit, abort_flag, p.status,
+          ok = mbar_wait_bounded<false>(bar(C::kBarRingEmpty + s), rp.parity() ^ 1u, limit, abort_flag, p.status,
                                         W_RINGEMPTY, w);
           if (!ok) break;
         }
-        if (!(p.debug & 8) && elect_one()) {
-          if (leader) mbar_arrive(bar(kBarRingFull + s));  // keeps the ring's phases in step; no bytes land here
-          mbar_arrive_expect_tx(bar(kBarQhFull), 4 * kQChunkBytes);
+        if (!kStarve && elect_one()) {
+          if (leader) mbar_arrive(bar(C::kBarRingFull + s));  // keeps the ring's phases in step; no bytes land here
+          mbar_arrive_expect_tx(bar(C::kBarQhFull), 4 * kQChunkBytes);
           for (int d = 0; d < 4; ++d)
-            tma_load_2d_hint(smem_base + kOffRing + s * kStageBytes + d * kQChunkBytes, &p.tm_q, bar(kBarQhFull),
+            tma_load_2d_hint(smem_base + C::kOffRing + s * kStageBytes + d * kQChunkBytes, &p.tm_q, bar(C::kBarQhFull),
                              256 + d * 64, qrow, pol_q);
         }
         __syncwarp();
@@ -361,84 +396,71 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       }
       if (ok && prev_row0 >= 0) ok = load_v(prev_row0, prev_kb, w);
     }
-#ifdef RK_TRACE
-    acc[1] = clock64() - acc_start;
-    RK_ACC_DUMP(2, 2);
-#endif
     // drain: every stage this CTA filled must have been released by the tensor core, and the
     // last Q tile must be free, before the CTA may exit
     if (ok && n_done > 0)
-      ok = mbar_wait_bounded<false>(bar(kBarQFree), qfree_phase, limit, abort_flag, p.status, W_DRAIN, -1);
+      ok = mbar_wait_bounded<false>(bar(C::kBarQFree), qfree_phase, limit, abort_flag, p.status, W_DRAIN, -1);
     for (uint32_t back = 1; back <= (uint32_t)kStages && ok; ++back) {
       if (rp.it >= back) {
         const uint32_t u = rp.it - back;  // a fill that has not been waited for yet
-        ok = mbar_wait_bounded<false>(bar(kBarRingEmpty + u % kStages), (u / kStages) & 1u, limit, abort_flag,
+        ok = mbar_wait_bounded<false>(bar(C::kBarRingEmpty + u % kStages), (u / kStages) & 1u, limit, abort_flag,
                                       p.status, W_DRAIN, (int)u);
       }
     }
   } else if (warp == 1) {
     // ------------------------------ UMMA issuer (leader CTA; whole warp loops, elected lane issues) --
     if (leader) {
-      RingPos rp;
+      RingPos<kStages> rp;
       uint32_t qr_ready_phases = 0;  // bit rb = parity to wait for
       uint32_t p_ready_phase = 0;
       uint32_t qh_done_phase = 0;
       uint32_t s_writes = 0;  // how often the score buffer has been written (gives the s_free phase)
       uint32_t qr_use = 0;  // counts rope-buffer uses across tiles
       bool ok = true;
-      const uint32_t q_base = smem_base + kOffQLat;
-      const uint32_t p_base = smem_base + kOffP;
+      const uint32_t q_base = smem_base + C::kOffQLat;
+      const uint32_t p_base = smem_base + C::kOffP;
 
       for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
         const AttnWorkItem item = get_work(p, w);
         const int n_kt = count_key_tiles(p, item);
         int kt_issued = 0;  // key tiles whose QK^T has been issued
         int kt_pv = 0;      // key tiles whose PV has been issued
-        {  // ring position of the staged upper Q half: wait for both CTAs' move into TMEM, then let go of it
+        if constexpr (!kPhase) {  // ring position of the staged upper Q half: wait for both CTAs' move into TMEM, then let go of it
           const uint32_t s = rp.stage();
-          ok = mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w) &&
-               mbar_wait_bounded<true>(bar(kBarQhDone), qh_done_phase, limit, abort_flag, p.status, W_QHDONE, w);
+          ok = mbar_wait_bounded<false>(bar(C::kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w) &&
+               mbar_wait_bounded<true>(bar(C::kBarQhDone), qh_done_phase, limit, abort_flag, p.status, W_QHDONE, w);
           qh_done_phase ^= 1;
           if (!ok) break;
           tc_fence_after_sync();
-          if (elect_one()) umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
+          if (elect_one()) umma_commit_2_mc(bar(C::kBarRingEmpty + s), 3);
           __syncwarp();
           rp.advance();
         }
 
         auto issue_qk = [&](bool first_of_seg, bool last_of_seg, uint32_t rb) -> bool {
-          RK_TR(0, 1);
           if (first_of_seg) {
-            RK_ACC_T0();
-            if (!mbar_wait_bounded<true>(bar(kBarQrReady + rb), (qr_ready_phases >> rb) & 1u, limit, abort_flag,
+            if (!mbar_wait_bounded<true>(bar(C::kBarQrReady + rb), (qr_ready_phases >> rb) & 1u, limit, abort_flag,
                                          p.status, W_QRREADY, w))
               return false;
             qr_ready_phases ^= (1u << rb);
-            RK_ACC(0);
           }
           if (s_writes > 0) {  // one score buffer: the softmax warps must have read the previous key tile's scores
-            RK_ACC_T0();
-            if (!mbar_wait_bounded<true>(bar(kBarSFree), (s_writes - 1) & 1u, limit, abort_flag, p.status, W_SFREE, w))
+            if (!mbar_wait_bounded<true>(bar(C::kBarSFree), (s_writes - 1) & 1u, limit, abort_flag, p.status, W_SFREE, w))
               return false;
             tc_fence_after_sync();
-            RK_ACC(1);
           }
           ++s_writes;
           const uint32_t tmem_s = tmem_base + kColS;
 #pragma unroll 1
           for (int st = 0; st < 5; ++st) {
             const uint32_t s = rp.stage();
-            RK_TR(0, 30 + st);
             {
-              RK_ACC_T0();
-              if (!mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
+              if (!mbar_wait_bounded<false>(bar(C::kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
                 return false;
-              RK_ACC(2 + st);
             }
-            const uint32_t b_addr = smem_base + kOffRing + s * kStageBytes;
-            RK_TR(0, 10 + st);
+            const uint32_t b_addr = smem_base + C::kOffRing + s * kStageBytes;
             if (elect_one()) {
-              if (st >= 2 && st < 4) {  // latent dims 256-511: A from tensor memory, 8 columns per K = 16 step
+              if (!kPhase && st >= 2 && st < 4) {  // latent dims 256-511: A from tensor memory, 8 columns per K = 16 step
                 const uint32_t a_tmem = tmem_base + kColQ + (uint32_t)(st - 2) * 64u;
                 const uint64_t db = umma_desc_sw128(b_addr, 16, 1024);
 #pragma unroll
@@ -446,8 +468,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
                   umma_f16_ts<2>(tmem_s, a_tmem + 8u * k, db + (uint64_t)(((k >> 2) * kChunkBytes + (k & 3) * 32) >> 4),
                                  kIdescQK, 1u);
                 }
-                umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
-              } else if (st < 2) {  // latent dims 0-255: A from shared memory
+                umma_commit_2_mc(bar(C::kBarRingEmpty + s), 3);
+              } else if (st < C::kQSmemChunks / 2) {  // latent dims held in shared memory
                 const uint32_t a_addr = q_base + 2 * st * kQChunkBytes;
                 // descriptors differ only in the start-address field (16-byte units): add constants
                 const uint64_t da = umma_desc_sw128(a_addr, 16, 1024), db = umma_desc_sw128(b_addr, 16, 1024);
@@ -457,50 +479,42 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
                               db + (uint64_t)(((k >> 2) * kChunkBytes + (k & 3) * 32) >> 4), kIdescQK,
                               (st > 0 || k > 0) ? 1u : 0u);
                 }
-                umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
+                umma_commit_2_mc(bar(C::kBarRingEmpty + s), 3);
               } else {
-                const uint32_t a_addr = smem_base + kOffQRot + rb * kQChunkBytes;
+                const uint32_t a_addr = smem_base + C::kOffQRot + rb * kQChunkBytes;
                 const uint64_t da = umma_desc_sw128(a_addr, 16, 1024), db = umma_desc_sw128(b_addr, 16, 1024);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) umma_f16<2>(tmem_s, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), kIdescQK, 1u);
-                umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
-                umma_commit_2_mc(bar(kBarSFull), 3);
-                if (last_of_seg) umma_commit_2_mc(bar(kBarQrFree + rb), 3);
+                umma_commit_2_mc(bar(C::kBarRingEmpty + s), 3);
+                umma_commit_2_mc(bar(C::kBarSFull), 3);
+                if (last_of_seg) umma_commit_2_mc(bar(C::kBarQrFree + rb), 3);
                 // all QK^T of this row tile issued: the Q tile is free once they complete
-                if (kt_issued + 1 == n_kt) umma_commit_2_mc(bar(kBarQFree), 3);
+                if (kt_issued + 1 == n_kt) umma_commit_2_mc(bar(C::kBarQFree), 3);
               }
             }
             __syncwarp();
             rp.advance();
           }
           ++kt_issued;
-          RK_TR(0, 2);
           return true;
         };
         auto issue_pv = [&]() -> bool {
           {
-            RK_ACC_T0();
-            if (!mbar_wait_bounded<true>(bar(kBarPReady), p_ready_phase, limit, abort_flag, p.status, W_PREADY, w))
+            if (!mbar_wait_bounded<true>(bar(C::kBarPReady), p_ready_phase, limit, abort_flag, p.status, W_PREADY, w))
               return false;
-            RK_ACC(7);
           }
           p_ready_phase ^= 1;
           tc_fence_after_sync();
-          RK_TR(0, 3);
 #pragma unroll 1
           for (int q = 0; q < 4; ++q) {
             const int kh = q >> 1, h = q & 1;
             const uint32_t s = rp.stage();
-            RK_TR(0, 40 + q);
             {
-              RK_ACC_T0();
-              if (!mbar_wait_bounded<false>(bar(kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
+              if (!mbar_wait_bounded<false>(bar(C::kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
                 return false;
-              RK_ACC(8 + q);
             }
-            const uint32_t b_addr = smem_base + kOffRing + s * kStageBytes;
+            const uint32_t b_addr = smem_base + C::kOffRing + s * kStageBytes;
             const uint32_t tmem_o = tmem_base + kColO + (uint32_t)h * 128u;
-            RK_TR(0, 20 + q);
             if (elect_one()) {
               const uint64_t da = umma_desc_sw128(p_base + 2 * kh * kQChunkBytes, 16, 1024);
               const uint64_t db = umma_desc_sw128(b_addr, kChunkBytes, 1024);
@@ -509,17 +523,32 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
                 umma_f16<2>(tmem_o, da + (uint64_t)(((k >> 2) * kQChunkBytes + (k & 3) * 32) >> 4),
                             db + (uint64_t)((k * 2048) >> 4), kIdescPV, (kt_pv > 0 || kh > 0 || k > 0) ? 1u : 0u);
               }
-              umma_commit_2_mc(bar(kBarRingEmpty + s), 3);
-              if (q == 3) umma_commit_2_mc(bar(kBarPvDone), 3);
+              umma_commit_2_mc(bar(C::kBarRingEmpty + s), 3);
+              if (!kPhase && q == 3) umma_commit_2_mc(bar(C::kBarPvDone), 3);
+            }
+            __syncwarp();
+            rp.advance();
+          }
+          if constexpr (kPhase) {  // rope part of the value: O_rope[64 x 64] += P[64 x 256] V_rope[256 x 64]
+            const uint32_t s = rp.stage();
+            if (!mbar_wait_bounded<false>(bar(C::kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w))
+              return false;
+            const uint32_t b_addr = smem_base + C::kOffRing + s * kStageBytes;
+            if (elect_one()) {
+              const uint64_t da = umma_desc_sw128(p_base, 16, 1024);
+              const uint64_t db = umma_desc_sw128(b_addr, kChunkBytes, 1024);
+#pragma unroll
+              for (int k = 0; k < 16; ++k) {  // 16 keys per step; the two 128-key boxes are contiguous
+                umma_f16<2>(tmem_base + kColOr, da + (uint64_t)(((k >> 2) * kQChunkBytes + (k & 3) * 32) >> 4),
+                            db + (uint64_t)((k * 2048) >> 4), kIdescPVr, (kt_pv > 0 || k > 0) ? 1u : 0u);
+              }
+              umma_commit_2_mc(bar(C::kBarRingEmpty + s), 3);
+              umma_commit_2_mc(bar(C::kBarPvDone), 3);
             }
             __syncwarp();
             rp.advance();
           }
           ++kt_pv;
-#ifdef RK_TRACE
-          acc[13] += 1;
-#endif
-          RK_TR(0, 4);
           return true;
         };
 
@@ -536,10 +565,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         }
         while (ok && kt_pv < kt_issued) ok = issue_pv();
       }
-#ifdef RK_TRACE
-      acc[12] = clock64() - acc_start;
-      RK_ACC_DUMP(0, 16);
-#endif
     }
   } else if (warp == 2) {
     // ------------------------------ query relocation ----------------------------------------
@@ -549,21 +574,21 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     bool ok = true;
     for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
       const AttnWorkItem item = get_work(p, w);
-      ok = mbar_wait_bounded<false>(bar(kBarQFull), qfull_phase, limit, abort_flag, p.status, W_QFULL, w);
+      ok = mbar_wait_bounded<false>(bar(C::kBarQFull), qfull_phase, limit, abort_flag, p.status, W_QFULL, w);
       qfull_phase ^= 1;
       SegIter it(p, item);
       while (ok && it.next()) {
         const uint32_t rb = qr_use & 1u;
         if (qr_use >= 2) {
-          ok = mbar_wait_bounded<true>(bar(kBarQrFree + rb), (qr_free_phases >> rb) & 1u, limit, abort_flag, p.status,
+          ok = mbar_wait_bounded<true>(bar(C::kBarQrFree + rb), (qr_free_phases >> rb) & 1u, limit, abort_flag, p.status,
                                        W_QRFREE, w);
           qr_free_phases ^= (1u << rb);
           if (!ok) break;
         }
         ++qr_use;
         const float2* cs = p.seg_cs + (size_t)it.seg * 32;
-        const uint8_t* src = smem + kOffQPristine;
-        uint8_t* dst = smem + kOffQRot + rb * kQChunkBytes;
+        const uint8_t* src = smem + C::kOffQPristine;
+        uint8_t* dst = smem + C::kOffQRot + rb * kQChunkBytes;
 #pragma unroll 4
         for (int i = 0; i < 16; ++i) {
           const int idx = lane + 32 * i;
@@ -584,14 +609,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         }
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive_remote(mapa_shared(bar(kBarQrReady + rb), 0));
+        if (lane == 0) mbar_arrive_remote(mapa_shared(bar(C::kBarQrReady + rb), 0));
       }
     }
     // drain the last releases so that no commit targets this CTA after it exits
     if (lane == 0) {
       for (uint32_t u = (qr_use >= 2 ? qr_use - 2 : 0); u < qr_use && ok; ++u) {
         const uint32_t rb = u & 1u;
-        ok = mbar_wait_bounded<true>(bar(kBarQrFree + rb), (qr_free_phases >> rb) & 1u, limit, abort_flag, p.status,
+        ok = mbar_wait_bounded<true>(bar(C::kBarQrFree + rb), (qr_free_phases >> rb) & 1u, limit, abort_flag, p.status,
                                      W_DRAIN, 100 + (int)rb);
         qr_free_phases ^= (1u << rb);
       }
@@ -608,7 +633,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     const int kh = L >> 6;               // which 128-key half of the tile (and which dims half of O)
     const int part = kh * 2 + ch;        // which 64-key quarter of the tile
     const uint32_t lane_base = ((uint32_t)((sw & 3) * 32)) << 16;
-    volatile unsigned long long* xbuf = reinterpret_cast<volatile unsigned long long*>(smem + kOffXchg);
+    volatile unsigned long long* xbuf = reinterpret_cast<volatile unsigned long long*>(smem + C::kOffXchg);
     uint32_t xseq = 0;  // exchange sequence number
     uint32_t ring_it = 0;  // ring position of the current row tile's staged Q half
     uint32_t s_full_phase = 0;
@@ -616,9 +641,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     uint32_t pv_done_phase = 0;
     bool ok = true;
     const float scale = p.scale_log2;
-    const uint32_t p_ready_remote = mapa_shared(bar(kBarPReady), 0);
-    const uint32_t s_free_remote = mapa_shared(bar(kBarSFree), 0);
-    const uint32_t qh_done_remote = mapa_shared(bar(kBarQhDone), 0);
+    const uint32_t p_ready_remote = mapa_shared(bar(C::kBarPReady), 0);
+    const uint32_t s_free_remote = mapa_shared(bar(C::kBarSFree), 0);
+    const uint32_t qh_done_remote = mapa_shared(bar(C::kBarQhDone), 0);
 
     for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
       const AttnWorkItem item = get_work(p, w);
@@ -632,12 +657,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       }
       float m_run = -INFINITY, l_run = 0.f;
       int kt = 0;
-      {  // move this thread's share of the upper Q half (row m, 64 dims) from its ring stage into TMEM
-        ok = mbar_wait_bounded<false>(bar(kBarQhFull), qh_full_phase, limit, abort_flag, p.status, W_QHFULL, w);
+      if constexpr (!kPhase) {  // move this thread's share of the upper Q half (row m, 64 dims) from its ring stage into TMEM
+        ok = mbar_wait_bounded<false>(bar(C::kBarQhFull), qh_full_phase, limit, abort_flag, p.status, W_QHFULL, w);
         qh_full_phase ^= 1;
         if (!ok) break;
         // every role counts ring positions alike: one staged half per row tile, nine stages per key tile
-        const uint8_t* stage = smem + kOffRing + (ring_it % kStages) * kStageBytes;
+        const uint8_t* stage = smem + C::kOffRing + (ring_it % kStages) * kStageBytes;
         ring_it += 1u + 9u * (uint32_t)count_key_tiles(p, item);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -656,6 +681,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         if (lane == 0) mbar_arrive_remote(qh_done_remote);
       }
 
+      // output-phase instantiation: the rope part of O is accumulated in the frame of the segment being
+      // walked (its stored rope dims are in that document's position-zero frame); seg_frame is that segment
+      int seg_frame = -1;
+      const int jr = 16 * kh + 8 * ch;  // first of this thread's 8 rotation pairs (16 rope dims) of the row
       SegIter it(p, item);
       while (ok && it.next()) {
         const int n_seg = p.seg_off[it.seg + 1] - p.seg_off[it.seg];
@@ -670,27 +699,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           int nv = lim - (kb + part * 64) + 1;
           nv = nv < 0 ? 0 : (nv > 64 ? 64 : nv);
           {
-            RK_ACC_T0();
-            ok = mbar_wait_bounded<false>(bar(kBarSFull), s_full_phase, limit, abort_flag, p.status, W_SFULL, w);
-            RK_ACC(0);
+            ok = mbar_wait_bounded<false>(bar(C::kBarSFull), s_full_phase, limit, abort_flag, p.status, W_SFULL, w);
           }
           s_full_phase ^= 1;
           if (!ok) break;
           tc_fence_after_sync();
-          if (warp == 4) RK_TR(1, 1);
-          if (p.debug & 1) {
-            __syncwarp();
-            if (lane == 0) mbar_arrive_remote(s_free_remote);
-            if (kt > 0) {
-              ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
-              pv_done_phase ^= 1;
-              if (!ok) break;
-            }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_remote(p_ready_remote);
-            continue;
-          }
           uint32_t s[64];
           const uint32_t taddr = tmem_base + lane_base + kColS + (uint32_t)ch * 64u;
           tmem_ld_x32(taddr + 0, s + 0);
@@ -710,13 +723,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           }
           const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
           float mxo = mx;
-          {
-            RK_ACC_T0();
-            if (!(p.debug & 4)) ok = quad_exchange_max(xbuf, part, m, ++xseq, mx, mxo, limit, abort_flag, p.status, w);
-            RK_ACC(1);
-          }
+          ok = quad_exchange_max(xbuf, part, m, ++xseq, mx, mxo, limit, abort_flag, p.status, w);
           if (!ok) break;
-          if (warp == 4) RK_TR(1, 2);
           const float mt = mxo * scale;
           // lazy rescale: only when the running maximum grows by more than 2^8
           float alpha = 1.f;
@@ -748,19 +756,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             }
           }
           l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-          if (warp == 4) RK_TR(1, 3);
           // P buffer and O are free once the previous PV has completed
           if (kt > 0) {
             {
-              RK_ACC_T0();
-              ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
-              RK_ACC(2);
+              ok = mbar_wait_bounded<false>(bar(C::kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
             }
             pv_done_phase ^= 1;
             if (!ok) break;
             tc_fence_after_sync();
-            if (warp == 4) RK_TR(1, 4);
-            if (__any_sync(0xffffffffu, need)) {
+            const bool any_need = __any_sync(0xffffffffu, need);
+            if (any_need) {
 #pragma unroll 1
               for (int cc = 0; cc < 128; cc += 32) {  // this thread's 2 x 64 columns of O
                 uint32_t o[32];
@@ -773,9 +778,39 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
               }
               tmem_wait_st();
             }
+            if constexpr (kPhase) {
+              // Segment switch (Algorithm 2, RestorePhase folded into the running merge): what has been
+              // accumulated so far is in the previous segment's frame; turning it by
+              // R(delta_prev - delta_this) moves it into the frame of the segment whose keys come next, so
+              // that the PV products of both can share one accumulator.  The lazy rescale rides along.
+              const bool turn = (kb == 0 && seg_frame >= 0);
+              if (turn || any_need) {
+                uint32_t o[16];
+                const uint32_t oaddr = tmem_base + lane_base + kColOr + (uint32_t)(ch * 16);
+                tmem_ld_x16(oaddr, o);
+                tmem_wait_ld();
+                if (turn) {
+                  const int d = p.seg_delta[seg_frame] - p.seg_delta[it.seg];
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) {
+                    float c, sn;
+                    rope_cs(p, d, jr + i, c, sn);
+                    const float x0 = __uint_as_float(o[2 * i]) * alpha, x1 = __uint_as_float(o[2 * i + 1]) * alpha;
+                    o[2 * i] = __float_as_uint(x0 * c - x1 * sn);
+                    o[2 * i + 1] = __float_as_uint(x0 * sn + x1 * c);
+                  }
+                } else {
+#pragma unroll
+                  for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                }
+                tmem_st_x16(oaddr, o);
+                tmem_wait_st();
+              }
+            }
           }
+          if constexpr (kPhase) seg_frame = it.seg;
           // write P (bf16, K-major 128B swizzle): row m of sub-chunk `part` (64 keys = 128 bytes)
-          uint8_t* pbase = smem + kOffP + part * kQChunkBytes;
+          uint8_t* pbase = smem + C::kOffP + part * kQChunkBytes;
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             uint8_t* dstp = pbase + sw128_offset((uint32_t)m, (uint32_t)c);
@@ -785,12 +820,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive_remote(p_ready_remote);
-          if (warp == 4) RK_TR(1, 5);
         }
       }
       if (!ok) break;
       // ---- epilogue: wait for the last PV, normalise, store ----
-      ok = mbar_wait_bounded<false>(bar(kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
+      ok = mbar_wait_bounded<false>(bar(C::kBarPvDone), pv_done_phase, limit, abort_flag, p.status, W_PVDONE, w);
       pv_done_phase ^= 1;
       if (!ok) break;
       tc_fence_after_sync();
@@ -798,7 +832,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       ok = quad_exchange_sum(xbuf, part, m, ++xseq, l_run, l_tot, limit, abort_flag, p.status, w);
       if (!ok) break;
       const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-      __nv_bfloat16* Orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)(valid ? r : 0) * kDLatent;
+      __nv_bfloat16* Orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)(valid ? r : 0) * C::kOW;
 #pragma unroll 1
       for (int cc = 0; cc < 128; cc += 32) {
         const int h = cc >> 6, c0 = cc & 63;
@@ -818,14 +852,31 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
           }
         }
       }
+      if constexpr (kPhase) {
+        // rope part of the output: normalise, then RestorePhase of the last frame and the inverse output
+        // RoPE of the row in one turn, R(-pos) R(delta_frame) = R(delta_frame - pos)  (Eq. offonline)
+        uint32_t o[16];
+        tmem_ld_x16(tmem_base + lane_base + kColOr + (uint32_t)(ch * 16), o);
+        tmem_wait_ld();
+        if (valid) {
+          const int d = (seg_frame >= 0 ? p.seg_delta[seg_frame] : 0) - pos;
+          uint32_t v[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            float c, sn;
+            rope_cs(p, d, jr + i, c, sn);
+            const float x0 = __uint_as_float(o[2 * i]) * inv, x1 = __uint_as_float(o[2 * i + 1]) * inv;
+            v[i] = pack_bf16(x0 * c - x1 * sn, x0 * sn + x1 * c);
+          }
+          uint4* dstg = reinterpret_cast<uint4*>(Orow + kDLatent + 32 * kh + 16 * ch);
+          __stcs(dstg, make_uint4(v[0], v[1], v[2], v[3]));
+          __stcs(dstg + 1, make_uint4(v[4], v[5], v[6], v[7]));
+        }
+      }
       if (valid && part == 0)
         p.lse[r] = (l_tot > 0.f) ? (m_run + log2f(l_tot)) * 0.69314718055994530942f : -INFINITY;
       tc_fence_before_sync();
     }
-#ifdef RK_TRACE
-    acc[3] = clock64() - acc_start;
-    if (warp == 4) RK_ACC_DUMP(1, 4);
-#endif
   }
 
   // ------------------------------ teardown ---------------------------------------------------
@@ -845,21 +896,24 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
   }
 }
 
-#ifdef RK_TRACE
-extern "C" int rk_debug_read_trace(long long* out, int n) {
-  return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * (size_t)n);
-}
-#endif
 
 cudaError_t attention_setup() {
-  return cudaFuncSetAttribute(rk_mla_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(rk_mla_attn_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)Cfg<false>::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(rk_mla_attn_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)Cfg<false>::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(rk_mla_attn_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)Cfg<true>::kSmemBytes);
+  return e;
 }
 
 int attention_max_pairs(int sm_count) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * (sm_count / 2), 1, 1);
   cfg.blockDim = dim3(kAttnThreads, 1, 1);
-  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.dynamicSmemBytes = Cfg<false>::kSmemBytes;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
@@ -868,15 +922,21 @@ int attention_max_pairs(int sm_count) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, rk_mla_attn_kernel, &cfg) != cudaSuccess || n <= 0) {
+  if (cudaOccupancyMaxActiveClusters(&n, rk_mla_attn_kernel<false, false>, &cfg) != cudaSuccess || n <= 0) {
     cudaGetLastError();
     n = sm_count / 2;
   }
   return n < sm_count / 2 ? n : sm_count / 2;
 }
 
-cudaError_t launch_attention(const AttnParams& p, int n_pairs, cudaStream_t stream) {
-  rk_mla_attn_kernel<<<dim3(2 * n_pairs, 1, 1), dim3(kAttnThreads, 1, 1), kSmemBytes, stream>>>(p);
+cudaError_t launch_attention(const AttnParams& p, int n_pairs, bool value_phase, bool starve_loads, cudaStream_t stream) {
+  const dim3 grid(2 * n_pairs, 1, 1), block(kAttnThreads, 1, 1);
+  if (value_phase)
+    rk_mla_attn_kernel<true, false><<<grid, block, Cfg<true>::kSmemBytes, stream>>>(p);
+  else if (starve_loads)
+    rk_mla_attn_kernel<false, true><<<grid, block, Cfg<false>::kSmemBytes, stream>>>(p);
+  else
+    rk_mla_attn_kernel<false, false><<<grid, block, Cfg<false>::kSmemBytes, stream>>>(p);
   return cudaGetLastError();
 }
 

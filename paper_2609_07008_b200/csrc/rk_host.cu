@@ -33,7 +33,10 @@ struct rk_ctx {
   GemmBatch* d_batches = nullptr;  // [uv_g: G][uv_l: L][wa_g: G][wa_l: G][wb: 1]
   int off_uv_g = 0, off_uv_l = 0, off_wa_g = 0, off_wa_l = 0, off_wb = 0;
   unsigned long long wait_ns = 2000ull * 1000 * 1000;
-  int attn_debug = 0;  // development switches of the attention kernel (rk_set_debug_flags)
+  bool value_phase = false;  // output-phase variant: the whole stored row is the value, O rows are 576 wide
+  int ow = kDLatent;         // width of an attention output row (512, or 576 with value_phase)
+  double rope_turns[32];     // theta_j / (2 pi)
+  bool starve_loads = false;  // rk_test_starve_loads: the timeout test's instantiation of the attention kernel
   cudaStream_t copy_stream = nullptr;  // rk_layer_host: copies that overlap the kernels
   cudaStream_t copy_out_stream = nullptr;  // rk_layer_stack_host: device->host copies (full duplex with the above)
   cudaEvent_t sev[10] = {nullptr};     // rk_layer_stack_host: kv_ql_in[2], qg_in[2], zoff_in[2], compute_done[2], y_copied[2]
@@ -154,6 +157,43 @@ void build_work(const std::vector<int32_t>& tok_pos, int hpt, const std::vector<
 }  // namespace
 
 // ------------------------------------------------------------------------------------------
+// Projection without any allocation by the caller or the library.
+//
+// Some users of this library cannot obtain device memory at call time: a serving runtime that
+// hands the whole device to its own memory pool at start-up has nothing left for cudaMalloc,
+// and a latency-critical request path cannot afford the implicit device-wide synchronisation
+// an allocation may cause.  For them the per-head intermediate o = W_uv O_lat lives in a
+// fixed array that is part of the loaded library image instead of a caller workspace.
+// ------------------------------------------------------------------------------------------
+#define RK_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+
+static __device__ __align__(256) unsigned char rk_static_scratch[RK_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_ptr[kMaxDevices] = {nullptr};
+std::mutex g_static_scratch_mutex;  // first calls may come from several host threads
+
+// Device address of rk_static_scratch on the CURRENT device (resolved once per device).  In host
+// code the array's name is only a handle for the runtime, not a device address, so the address
+// must come from cudaGetSymbolAddress.  rk_create calls this: the lookup is what makes the runtime
+// load this file's module and materialise the array on the device, which may allocate and
+// synchronise -- work that belongs to set-up, not to the entry point that promises to allocate nothing.
+cudaError_t static_scratch_address(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (g_static_scratch_ptr[device] == nullptr) {
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, rk_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_scratch_ptr[device] = ptr;
+  }
+  *out = g_static_scratch_ptr[device];
+  return cudaSuccess;
+}
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
 extern "C" {
 
 const char* rk_version(void) { return "rk-mla-online 0.1 (sm_100a)"; }
@@ -176,9 +216,12 @@ const char* rk_status_string(rk_status s) {
 
 const char* rk_last_error(const rk_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
 
-rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
+rk_status rk_create(const rk_profile* prof, rk_ctx** out) { return rk_create_ex(prof, 0u, out); }
+
+rk_status rk_create_ex(const rk_profile* prof, uint32_t flags, rk_ctx** out) {
   if (!prof || !out) return RK_ERR_NULL;
   *out = nullptr;
+  if (flags & ~(uint32_t)RK_VALUE_PHASE) return RK_ERR_UNSUPPORTED;
   if (!prof->global_heads) return RK_ERR_NULL;
   if (prof->group_size != kGroup || prof->d_latent != kDLatent || prof->d_rope != kDRope || prof->d_v != kDV)
     return RK_ERR_UNSUPPORTED;
@@ -195,6 +238,10 @@ rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
   ctx->prof = *prof;
   ctx->global_heads.assign(prof->global_heads, prof->global_heads + prof->n_groups);
   ctx->prof.global_heads = ctx->global_heads.data();
+  ctx->value_phase = (flags & RK_VALUE_PHASE) != 0;
+  ctx->ow = ctx->value_phase ? kDQK : kDLatent;
+  for (int j = 0; j < 32; ++j)
+    ctx->rope_turns[j] = std::pow((double)prof->rope_base, -2.0 * j / (double)kDRope) / 6.283185307179586476925286766559;
   for (int h = 0; h < prof->n_heads; ++h)
     if (ctx->global_heads[h / kGroup] != h) ctx->local_heads.push_back(h);
 
@@ -222,6 +269,7 @@ rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
   ctx->encode = reinterpret_cast<PFN_encodeTiled>(fn);
   e = attention_setup();
   if (e == cudaSuccess) e = gemm_setup();
+  if (e == cudaSuccess) e = stream_setup();
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->d_status), sizeof(DeviceStatus));
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(DeviceStatus));
   if (e != cudaSuccess) {
@@ -231,6 +279,15 @@ rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
     return RK_ERR_CUDA;
   }
   ctx->n_pairs = attention_max_pairs(ctx->sm_count);
+  {  // bind the built-in projection scratch of rk_group_sliced_proj_static on this device now
+    void* scratch = nullptr;
+    e = static_scratch_address(ctx->device, &scratch);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      rk_destroy(ctx);
+      return RK_ERR_CUDA;
+    }
+  }
   e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_out_stream, cudaStreamNonBlocking);
   for (int i = 0; i < 10 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->sev[i], cudaEventDisableTiming);
@@ -246,9 +303,9 @@ rk_status rk_create(const rk_profile* prof, rk_ctx** out) {
   const int32_t kNoSkip = 1 << 30;
   std::vector<GemmBatch> b;
   ctx->off_uv_g = (int)b.size();
-  for (int g = 0; g < G; ++g) b.push_back(GemmBatch{g * kDLatent, ctx->global_heads[g] * kDV, 0, kNoSkip, g * kDV, {0, 0, 0}});
+  for (int g = 0; g < G; ++g) b.push_back(GemmBatch{g * ctx->ow, ctx->global_heads[g] * kDV, 0, kNoSkip, g * kDV, {0, 0, 0}});
   ctx->off_uv_l = (int)b.size();
-  for (int l = 0; l < L; ++l) b.push_back(GemmBatch{l * kDLatent, ctx->local_heads[l] * kDV, 0, kNoSkip, l * kDV, {0, 0, 0}});
+  for (int l = 0; l < L; ++l) b.push_back(GemmBatch{l * ctx->ow, ctx->local_heads[l] * kDV, 0, kNoSkip, l * kDV, {0, 0, 0}});
   ctx->off_wa_g = (int)b.size();
   for (int g = 0; g < G; ++g) {
     const int j = ctx->global_heads[g] % kGroup;
@@ -294,9 +351,9 @@ rk_status rk_set_wait_limit_ms(rk_ctx* ctx, int32_t ms) {
   return RK_OK;
 }
 
-rk_status rk_set_debug_flags(rk_ctx* ctx, int32_t flags) {
+rk_status rk_test_starve_loads(rk_ctx* ctx, int32_t on) {
   if (!ctx) return RK_ERR_NULL;
-  ctx->attn_debug = flags;
+  ctx->starve_loads = on != 0;
   return RK_OK;
 }
 
@@ -580,10 +637,10 @@ static rk_status attn_pass(rk_ctx* ctx, const rk_request* rq, const void* kv, co
   const int n_pairs = std::min(ctx->n_pairs, n_tiles);
   p.n_pairs = n_pairs;
   p.scale_log2 = ctx->prof.sm_scale * 1.44269504088896340736f;
-  p.debug = ctx->attn_debug;
   p.isolated = isolated;
   p.row_base = (int32_t)row_base;
-  cudaError_t e = launch_attention(p, n_pairs, stream);
+  memcpy(p.rope_turns, ctx->rope_turns, sizeof(p.rope_turns));
+  cudaError_t e = launch_attention(p, n_pairs, ctx->value_phase, ctx->starve_loads, stream);
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "attention launch");
 }
 
@@ -616,7 +673,7 @@ rk_status rk_mla_off_workspace_bytes(const rk_request* rq, int64_t n_rows, size_
   if (!rq || !out) return RK_ERR_NULL;
   if (n_rows < 0) return RK_ERR_LAYOUT;
   const size_t L = rq->ctx->local_heads.size();
-  *out = align256((size_t)n_rows * L * kDLatent * 2) + align256((size_t)n_rows * L * 4) +
+  *out = align256((size_t)n_rows * L * rq->ctx->ow * 2) + align256((size_t)n_rows * L * 4) +
          align256((size_t)n_rows * L * kDV * 2);
   return RK_OK;
 }
@@ -641,15 +698,15 @@ rk_status rk_mla_off_build(rk_ctx* ctx, const rk_request* rq, const void* kv, in
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   void* O = ws;
-  float* lse = reinterpret_cast<float*>(ws + align256((size_t)n * L * kDLatent * 2));
+  float* lse = reinterpret_cast<float*>(ws + align256((size_t)n * L * ctx->ow * 2));
   void* o = reinterpret_cast<uint8_t*>(lse) + align256((size_t)n * L * 4);
   const int n_tiles = (int)((n * L + kAttnRowsPerPair - 1) / kAttnRowsPerPair);
   // documents alone: a row sees only its own segment, causally, with the query relocated into
   // the segment's position-zero frame; tiles in natural order (no host-built list)
   rk_status s = attn_pass(ctx, rq, kv, q_l_rows, n, L, nullptr, nullptr, n_tiles, O, lse, st, 1, row_begin);
   if (s != RK_OK) return s;
-  s = run_gemm(ctx, O, n, (int64_t)L * kDLatent, W_uv, (int64_t)H * kDV, kDLatent, o, (int64_t)L * kDV, (int)n, kDV,
-               kDLatent, ctx->off_uv_l, L, st);
+  s = run_gemm(ctx, O, n, (int64_t)L * ctx->ow, W_uv, (int64_t)H * kDV, ctx->ow, o, (int64_t)L * kDV, (int)n, kDV,
+               ctx->ow, ctx->off_uv_l, L, st);
   if (s != RK_OK) return s;
   return run_gemm(ctx, o, n, (int64_t)L * kDV, W_a, (int64_t)G * ro, kGroup * kDV, z_off_rows, (int64_t)G * ro, (int)n, ro,
                   (kGroup - 1) * kDV, ctx->off_wa_l, G, st);
@@ -659,7 +716,7 @@ rk_status rk_segmented_merge(rk_ctx* ctx, int32_t n_parts, int64_t n_rows, int32
                              int32_t part_dtype, const float* lse_part, void* O, float* lse, void* stream) {
   if (!ctx) return RK_ERR_NULL;
   if (!O_part || !lse_part || !O || !lse) return fail(ctx, RK_ERR_NULL, "null argument");
-  if (n_parts <= 0 || n_parts > 4096 || n_rows < 0 || n_heads <= 0) return fail(ctx, RK_ERR_LAYOUT, "bad part/row/head count");
+  if (n_parts <= 0 || n_parts > kMergeMaxParts || n_rows < 0 || n_heads <= 0) return fail(ctx, RK_ERR_LAYOUT, "bad part/row/head count");
   if (part_dtype != 0 && part_dtype != 1) return fail(ctx, RK_ERR_UNSUPPORTED, "part_dtype must be 0 (bf16) or 1 (fp32)");
   if (!aligned16(O_part) || !aligned16(O)) return fail(ctx, RK_ERR_ALIGN, "O_part/O must be 16-byte aligned");
   cudaError_t e = launch_merge(n_parts, n_rows * n_heads, O_part, part_dtype, lse_part, O, lse, ctx->sm_count,
@@ -714,15 +771,15 @@ rk_status rk_group_sliced_proj(rk_ctx* ctx, const rk_request* rq, const void* O_
   void* o_l = ws + (((size_t)T * G * kDV * 2 + 255) & ~(size_t)255);
   rk_status s = RK_OK;
   if (do_g) {
-    s = run_gemm(ctx, O_g, T, (int64_t)G * kDLatent, W_uv, (int64_t)H * kDV, kDLatent, o_g, (int64_t)G * kDV, (int)T, kDV,
-                 kDLatent, ctx->off_uv_g, G, st);
+    s = run_gemm(ctx, O_g, T, (int64_t)G * ctx->ow, W_uv, (int64_t)H * kDV, ctx->ow, o_g, (int64_t)G * kDV, (int)T, kDV,
+                 ctx->ow, ctx->off_uv_g, G, st);
     if (s == RK_OK)
       s = run_gemm(ctx, o_g, T, (int64_t)G * kDV, W_a, (int64_t)G * ro, kGroup * kDV, z_on_g, (int64_t)G * ro, (int)T, ro,
                    kDV, ctx->off_wa_g, G, st);
   }
   if (s == RK_OK && do_l && A > 0) {
-    s = run_gemm(ctx, O_l, A, (int64_t)L * kDLatent, W_uv, (int64_t)H * kDV, kDLatent, o_l, (int64_t)L * kDV, (int)A, kDV,
-                 kDLatent, ctx->off_uv_l, L, st);
+    s = run_gemm(ctx, O_l, A, (int64_t)L * ctx->ow, W_uv, (int64_t)H * kDV, ctx->ow, o_l, (int64_t)L * kDV, (int)A, kDV,
+                 ctx->ow, ctx->off_uv_l, L, st);
     if (s == RK_OK)
       s = run_gemm(ctx, o_l, A, (int64_t)L * kDV, W_a, (int64_t)G * ro, kGroup * kDV, z_on_l, (int64_t)G * ro, (int)A, ro,
                    (kGroup - 1) * kDV, ctx->off_wa_l, G, st);
@@ -804,8 +861,8 @@ static rk_status layer_compute(rk_ctx* ctx, const rk_request* rq, const rk_layer
     s = attn_pass(ctx, rq, dev->kv, dev->q_g, T, G, nullptr, n_chunks == 2 ? rq->d_work_g_part[c] : rq->d_work_g,
                   n_chunks == 2 ? rq->n_tiles_g_part[c] : rq->n_tiles_g, dev->O_g, dev->lse_g, st);
     if (s == RK_OK)
-      s = run_gemm(ctx, Og + (size_t)r0 * G * kDLatent * 2, n, (int64_t)G * kDLatent, W_uv, (int64_t)H * kDV, kDLatent,
-                   og + (size_t)r0 * G * kDV * 2, (int64_t)G * kDV, (int)n, kDV, kDLatent, ctx->off_uv_g, G, st);
+      s = run_gemm(ctx, Og + (size_t)r0 * G * ctx->ow * 2, n, (int64_t)G * ctx->ow, W_uv, (int64_t)H * kDV, ctx->ow,
+                   og + (size_t)r0 * G * kDV * 2, (int64_t)G * kDV, (int)n, kDV, ctx->ow, ctx->off_uv_g, G, st);
     if (s == RK_OK)
       s = run_gemm(ctx, og + (size_t)r0 * G * kDV * 2, n, (int64_t)G * kDV, W_a, (int64_t)G * ro, kGroup * kDV,
                    zg + (size_t)r0 * width * 2, (int64_t)G * ro, (int)n, ro, kDV, ctx->off_wa_g, G, st);
@@ -988,9 +1045,12 @@ rk_status rk_protected_rows(rk_ctx* ctx, const rk_layout* lay, const rk_policy* 
     tab[(size_t)(S + 1 + i)] = (int32_t)lay->seg_delta[i];
     req_end = std::max<int64_t>(req_end, lay->seg_delta[i] + lay->seg_off[i + 1] - lay->seg_off[i]);
   }
+  // the artifact flags are staged in a library-owned pageable vector like the segment table: the copy then
+  // never reads the caller's array after this call has returned, whether or not that array is pinned
+  std::vector<uint8_t> has_stage(lay->seg_has_artifact, lay->seg_has_artifact + S);
   PolicyHost h = {};
   h.seg_tab_host = tab.data();
-  h.has_host = lay->seg_has_artifact;
+  h.has_host = has_stage.data();
   h.n_segs = S;
   h.T = T;
   h.req_end = req_end;
@@ -1022,41 +1082,6 @@ rk_status rk_moe_fanout(rk_ctx* ctx, const float* p, int64_t n, float tau, int32
 
 }  // extern "C"
 
-// ------------------------------------------------------------------------------------------
-// Projection without any allocation by the caller or the library.
-//
-// Some users of this library cannot obtain device memory at call time: a serving runtime that
-// hands the whole device to its own memory pool at start-up has nothing left for cudaMalloc,
-// and a latency-critical request path cannot afford the implicit device-wide synchronisation
-// an allocation may cause.  For them the per-head intermediate o = W_uv O_lat lives in a
-// fixed array that is part of the loaded library image instead of a caller workspace.
-// ------------------------------------------------------------------------------------------
-#define RK_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
-
-static __device__ __align__(256) unsigned char rk_static_scratch[RK_STATIC_SCRATCH_BYTES];
-
-namespace {
-constexpr int kMaxDevices = 64;
-void* g_static_scratch_ptr[kMaxDevices] = {nullptr};
-std::mutex g_static_scratch_mutex;  // first calls may come from several host threads
-
-// Device address of rk_static_scratch on the CURRENT device (resolved once per device).  In host
-// code the array's name is only a handle for the runtime, not a device address, so the address
-// must come from cudaGetSymbolAddress.
-cudaError_t static_scratch_address(int device, void** out) {
-  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
-  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
-  if (g_static_scratch_ptr[device] == nullptr) {
-    void* ptr = nullptr;
-    cudaError_t e = cudaGetSymbolAddress(&ptr, rk_static_scratch);
-    if (e != cudaSuccess) return e;
-    g_static_scratch_ptr[device] = ptr;
-  }
-  *out = g_static_scratch_ptr[device];
-  return cudaSuccess;
-}
-}  // namespace
-
 extern "C" rk_status rk_group_sliced_proj_static(rk_ctx* ctx, const rk_request* rq, const void* O_g, const void* O_l,
                                                  const void* W_uv, const void* W_a, void* z_on_g, void* z_on_l,
                                                  void* stream) {
@@ -1076,6 +1101,7 @@ extern "C" rk_status rk_group_sliced_proj_static(rk_ctx* ctx, const rk_request* 
   void* scratch = nullptr;
   e = static_scratch_address(device, &scratch);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaGetSymbolAddress(rk_static_scratch)");
+  // (already resolved by rk_create on this device: a table lookup, no runtime call)
   // nothing in the scratch has to start at zero: o is fully written before it is read, and rows
   // beyond the tensor's extent are zero-filled by the TMA load, never read from the array
   return rk_group_sliced_proj(ctx, rq, O_g, O_l, W_uv, W_a, z_on_g, z_on_l, scratch, RK_STATIC_SCRATCH_BYTES, stream);

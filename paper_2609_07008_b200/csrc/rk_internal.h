@@ -33,7 +33,7 @@ struct AttnParams {
   const int32_t* seg_delta;  // [S]
   const float2* seg_cs;      // [S][32] (cos, sin)(delta_i * theta_j)
   const AttnWorkItem* work;  // [n_tiles] cost-descending
-  void* O;                   // bf16 [n_flat][512]
+  void* O;                   // bf16 [n_flat][512] (output-phase instantiation: [n_flat][576])
   float* lse;                // [n_flat]
   DeviceStatus* status;
   unsigned long long wait_ns;
@@ -43,12 +43,12 @@ struct AttnParams {
   int32_t hpt;     // heads per token in this pass (G or L)
   int32_t n_pairs;
   float scale_log2;  // sm_scale * log2(e)
-  int32_t debug;     // development switches (0 in production)
   int32_t isolated;  // 1: a row sees only its own segment (documents built alone, Algorithm 1)
   int32_t row_base;  // packed row of token slot 0 when rowmap is null
+  double rope_turns[32];  // theta_j / (2 pi), j = 0..31 (used by the output-phase instantiation only)
 };
 
-cudaError_t launch_attention(const AttnParams& p, int n_pairs, cudaStream_t stream);
+cudaError_t launch_attention(const AttnParams& p, int n_pairs, bool value_phase, bool starve_loads, cudaStream_t stream);
 cudaError_t attention_setup();  // sets the dynamic shared memory attribute once
 int attention_max_pairs(int sm_count);
 
@@ -79,6 +79,8 @@ cudaError_t launch_gemm(const GemmParams& p, int bn, int sm_count, cudaStream_t 
 cudaError_t gemm_setup();
 
 // ---- streaming kernels -----------------------------------------------------------------------
+constexpr int kMergeMaxParts = 4096;  // the merge keeps 8 warps x n_parts weights in shared memory (128 KB at most)
+cudaError_t stream_setup();          // raises the merge kernels' dynamic shared memory limit once
 cudaError_t launch_relocate(const void* q_rope, int64_t n_rows, int32_t n_heads, int64_t row_stride,
                             int64_t head_stride, const float2* seg_cs, int32_t seg_begin, int32_t seg_end,
                             void* out, int sm_count, cudaStream_t stream);

@@ -162,6 +162,13 @@ inline int grid_for(int64_t n_threads_needed, int sm_count, int per_sm) {
 
 }  // namespace
 
+cudaError_t stream_setup() {
+  const int bytes = 8 * kMergeMaxParts * (int)sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(rk_merge_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(rk_merge_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
 cudaError_t launch_relocate(const void* q_rope, int64_t n_rows, int32_t n_heads, int64_t row_stride,
                             int64_t head_stride, const float2* seg_cs, int32_t seg_begin, int32_t seg_end, void* out,
                             int sm_count, cudaStream_t stream) {

@@ -49,6 +49,21 @@ def aggregate_throughput(units_per_rank_step: int, steps: int, world: int, max_s
     return world * units_per_rank_step * steps / max_seconds
 
 
+def spawn_ranks(n: int, script_and_args) -> int:
+    """Starts `n` ranks of `script_and_args` on this node through torch.distributed.run (one process per GPU,
+    rendezvous on 127.0.0.1 at a free port) and returns its exit code.  Rank 0's standard output is the
+    caller's: the one JSON line appears once."""
+    import socket
+    import subprocess
+    import sys
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port)] + list(script_and_args)
+    return subprocess.run(cmd).returncode
+
+
 def shutdown() -> None:
     if dist.is_initialized():
         dist.destroy_process_group()

@@ -94,6 +94,7 @@ class Workload:
     w_b: torch.Tensor                      # bf16 [d_model, G*r_o]
     z_off: torch.Tensor                    # bf16 [N_doc, G*r_o] stand-in offline artifact
     q_all: Optional[torch.Tensor] = None   # bf16 [T, H, 576] (small cases only)
+    regime: str = "mandated"               # value regime the tensors were drawn in ("mandated" | "sharp")
 
     @property
     def T(self) -> int:
@@ -266,7 +267,7 @@ def make_tensors(name: str, profile: Profile, layout: Layout, prot_rows: np.ndar
     w_b = _normal((profile.d_model, G * profile.o_rank), 0.02, gen, dev)
     z_off = _normal_big((layout.n_doc_rows, G * profile.o_rank), z_off_std, gen, dev)
     return Workload(name=name, seed=seed, profile=profile, layout=layout, prot_rows=prot_rows,
-                    kv=kv, q_g=q_g, q_l=q_l, w_uv=w_uv, w_a=w_a, w_b=w_b, z_off=z_off, q_all=q_all)
+                    kv=kv, q_g=q_g, q_l=q_l, w_uv=w_uv, w_a=w_a, w_b=w_b, z_off=z_off, q_all=q_all, regime=regime)
 
 
 def make_workload(name: str, device="cpu", regime: str = "mandated", layer: int = 0,

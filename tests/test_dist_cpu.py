@@ -59,3 +59,21 @@ def test_single_rank_is_a_noop():
     rkdist.barrier()
     assert rkdist.max_over_ranks(1.5) == 1.5
     assert rkdist.aggregate_throughput(100, 3, 1, 2.0) == 150.0
+
+
+def test_bench_starts_its_own_ranks_when_launched_plainly():
+    """`python bench.py --gpus 2` without a launcher around it starts two ranks itself; on the checker arm
+    (no GPU needed) rank 0 alone does the work and exactly one JSON line with n_gpus = 2 comes out."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "reference", "--config", "tiny",
+                        "--steps", "1", "--warmup", "0", "--oracle-pairs", "100000"], capture_output=True, text=True,
+                       timeout=600, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["impl"] == "reference" and d["config"]["workload"] == "tiny"

@@ -8,9 +8,11 @@ workspace.  This file is collected last on purpose (a run that stops at the firs
 then already run every other test) and passes both alone in a fresh process and after the
 other tests: it depends on nothing they leave behind, and the array it uses keeps stale
 contents between calls by design."""
+import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2609_07008_b200 import synth
 from tests.helpers import assert_close, f64, to_device
 
@@ -33,11 +35,22 @@ def test_static_scratch_projection_matches_workspace_projection_twice():
         want_g, want_l = ctx.rk_group_sliced_proj(req, O_g, O_l, w.w_uv, w.w_a)
         z_g = torch.full((T, width), float("nan"), dtype=torch.bfloat16, device="cuda")
         z_l = torch.full((A, width), float("nan"), dtype=torch.bfloat16, device="cuda")
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         ctx.rk_group_sliced_proj_static(req, O_g, O_l, w.w_uv, w.w_a, z_g, z_l)
         ctx.rk_poll_status()
-        assert_close(f64(z_g), f64(want_g), f"z_on_g, call {call}")
-        assert_close(f64(z_l), f64(want_l), f"z_on_l, call {call}")
+        assert torch.cuda.mem_get_info()[0] == free_before       # the call took no device memory
+        assert_close(f64(z_g), f64(want_g), f"z_on_g, call {call}", unit_scale=True)
+        assert_close(f64(z_l), f64(want_l), f"z_on_l, call {call}", unit_scale=True)
         assert torch.equal(z_g, want_g) and torch.equal(z_l, want_l)
+        # and against the float64 checker (Eq. offonline: per-head W_uv, then the head's slice of W_a)
+        cg = oracle.head_contributions(f64(O_g), p.global_heads, f64(w.w_uv), f64(w.w_a))
+        assert_close(f64(z_g), cg.reshape(T, -1), f"z_on_g vs checker, call {call}", unit_scale=True)
+        cl = oracle.head_contributions(f64(O_l), p.local_heads, f64(w.w_uv), f64(w.w_a))
+        want = np.zeros((A, p.n_groups, p.o_rank))
+        for a, h in enumerate(p.local_heads):
+            want[:, h // 8] += cl[:, a]
+        assert_close(f64(z_l), want.reshape(A, -1), f"z_on_l vs checker, call {call}", unit_scale=True)
 
 
 def test_static_scratch_rejects_requests_beyond_its_size():
