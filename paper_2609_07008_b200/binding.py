@@ -54,7 +54,7 @@ class rk_layer_io(C.Structure):
 
 
 EXPORTS = ["rk_version", "rk_status_string", "rk_create", "rk_destroy", "rk_last_error", "rk_poll_status",
-           "rk_set_wait_limit_ms", "rk_test_starve_loads", "rk_request_create", "rk_request_destroy", "rk_check_request",
+           "rk_create_ex", "rk_segmented_merge_phase", "rk_set_wait_limit_ms", "rk_test_starve_loads", "rk_request_create", "rk_request_destroy", "rk_check_request",
            "rk_request_get_info", "rk_workspace_bytes", "rk_relocate_q", "rk_mla_online_attn",
            "rk_segmented_merge", "rk_group_sliced_proj", "rk_group_sliced_proj_static", "rk_combine_offline",
            "rk_layer_host", "rk_layer_stack_host", "rk_mla_off_workspace_bytes", "rk_mla_off_build",
@@ -78,6 +78,8 @@ def _load() -> C.CDLL:
     lib.rk_poll_status.argtypes = [vp, vp]
     lib.rk_set_wait_limit_ms.argtypes = [vp, i32]
     lib.rk_test_starve_loads.argtypes = [vp, i32]
+    lib.rk_create_ex.argtypes = [C.POINTER(rk_profile), C.c_uint32, C.POINTER(vp)]
+    lib.rk_segmented_merge_phase.argtypes = [vp, vp, i32, i32, i64, i32, vp, i32, vp, vp, vp, vp, vp]
     lib.rk_request_create.argtypes = [vp, C.POINTER(rk_layout), C.POINTER(i32), i64, C.POINTER(vp)]
     lib.rk_request_destroy.argtypes = [vp]
     lib.rk_check_request.argtypes = [C.POINTER(rk_layout), C.POINTER(i32), i64, C.c_char_p, C.c_size_t]
@@ -153,21 +155,25 @@ class Context:
     """rk_ctx: one per (device, head profile)."""
 
     def __init__(self, n_heads, n_groups, o_rank, d_model, global_heads, sm_scale, rope_base=10000.0,
-                 group_size=8, d_latent=512, d_rope=64, d_v=128):
+                 group_size=8, d_latent=512, d_rope=64, d_v=128, value_phase=False):
         gh = np.ascontiguousarray(global_heads, dtype=np.int32)
         self._gh = gh
         self.profile = rk_profile(n_heads, n_groups, group_size, d_latent, d_rope, d_v, o_rank, d_model,
                                   float(sm_scale), float(rope_base), gh.ctypes.data_as(C.POINTER(C.c_int32)))
         self.handle = C.c_void_p()
-        s = lib.rk_create(C.byref(self.profile), C.byref(self.handle))
+        # value_phase: the output-phase variant (RK_VALUE_PHASE): attention outputs are 576 wide, W_uv [H,128,576]
+        s = lib.rk_create_ex(C.byref(self.profile), 1 if value_phase else 0, C.byref(self.handle))
         if s != RK_OK:
             raise RKError(s, "rk_create failed")
+        self.value_phase = bool(value_phase)
+        self.ow = 576 if value_phase else 512
         self.n_heads, self.n_groups, self.n_local = n_heads, n_groups, n_heads - n_groups
         self.o_rank, self.d_model = o_rank, d_model
 
     @classmethod
-    def from_profile(cls, p):
-        return cls(p.n_heads, p.n_groups, p.o_rank, p.d_model, p.global_heads, p.sm_scale, p.rope_base)
+    def from_profile(cls, p, value_phase=False):
+        return cls(p.n_heads, p.n_groups, p.o_rank, p.d_model, p.global_heads, p.sm_scale, p.rope_base,
+                   value_phase=value_phase)
 
     def check(self, s: int):
         if s != RK_OK:
@@ -213,10 +219,10 @@ class Context:
     def rk_mla_online_attn(self, req, kv, q_g, q_l, O_g=None, lse_g=None, O_l=None, lse_l=None):
         dev = kv.device
         if q_g is not None and O_g is None:
-            O_g = _empty((req.T, self.n_groups, 512), dtype=torch.bfloat16, device=dev)
+            O_g = _empty((req.T, self.n_groups, self.ow), dtype=torch.bfloat16, device=dev)
             lse_g = _empty((req.T, self.n_groups), dtype=torch.float32, device=dev)
         if q_l is not None and O_l is None:
-            O_l = _empty((req.A, self.n_local, 512), dtype=torch.bfloat16, device=dev)
+            O_l = _empty((req.A, self.n_local, self.ow), dtype=torch.bfloat16, device=dev)
             lse_l = _empty((req.A, self.n_local), dtype=torch.float32, device=dev)
         self.check(lib.rk_mla_online_attn(self.handle, req.handle, _ptr(kv), _ptr(q_g), _ptr(q_l), _ptr(O_g),
                                           _ptr(lse_g), _ptr(O_l), _ptr(lse_l), _stream()))
@@ -231,6 +237,20 @@ class Context:
             lse = _empty((n_rows, n_heads), dtype=torch.float32, device=O_part.device)
         self.check(lib.rk_segmented_merge(self.handle, P, n_rows, n_heads, _ptr(O_part), dt, _ptr(lse_part),
                                           _ptr(O), _ptr(lse), _stream()))
+        return O, lse
+
+    def rk_segmented_merge_phase(self, req, seg_begin: int, O_part: torch.Tensor, lse_part: torch.Tensor,
+                                 row_pos: Optional[torch.Tensor] = None, O=None, lse=None):
+        """Output-phase merge: part j belongs to segment seg_begin + j; O_part [P, n_rows, n_heads, 576]."""
+        P, n_rows, n_heads, d = O_part.shape
+        assert d == 576 and lse_part.shape == (P, n_rows, n_heads) and lse_part.dtype == torch.float32
+        assert row_pos is None or (row_pos.dtype == torch.int32 and row_pos.shape == (n_rows,))
+        dt = {torch.bfloat16: 0, torch.float32: 1}[O_part.dtype]
+        if O is None:
+            O = _empty((n_rows, n_heads, 576), dtype=torch.bfloat16, device=O_part.device)
+            lse = _empty((n_rows, n_heads), dtype=torch.float32, device=O_part.device)
+        self.check(lib.rk_segmented_merge_phase(self.handle, req.handle, seg_begin, P, n_rows, n_heads, _ptr(O_part), dt,
+                                                _ptr(lse_part), _ptr(row_pos), _ptr(O), _ptr(lse), _stream()))
         return O, lse
 
     def rk_group_sliced_proj(self, req, O_g, O_l, W_uv, W_a, z_on_g=None, z_on_l=None, workspace=None):
@@ -321,7 +341,7 @@ class Context:
         bf, f32 = torch.bfloat16, torch.float32
         e = lambda shape, dt=bf: _empty(shape, dtype=dt, device=device)
         return dict(kv=e((T, 576)), q_g=e((T, G, 576)), q_l=e((max(A, 1), L, 576)),
-                    z_off=e((max(req.n_off_rows, 1), width)), O_g=e((T, G, 512)), O_l=e((max(A, 1), L, 512)),
+                    z_off=e((max(req.n_off_rows, 1), width)), O_g=e((T, G, self.ow)), O_l=e((max(A, 1), L, self.ow)),
                     z_on_g=e((T, width)), z_on_l=e((max(A, 1), width)), z=e((T, width)), y=e((T, self.d_model)),
                     lse_g=e((T, G), f32), lse_l=e((max(A, 1), L), f32),
                     workspace=_empty(max(req.workspace_bytes, 256), dtype=torch.uint8, device=device))

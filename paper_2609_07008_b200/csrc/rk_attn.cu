@@ -663,7 +663,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         if (!ok) break;
         // every role counts ring positions alike: one staged half per row tile, nine stages per key tile
         const uint8_t* stage = smem + C::kOffRing + (ring_it % kStages) * kStageBytes;
-        ring_it += 1u + 9u * (uint32_t)count_key_tiles(p, item);
+        ring_it += 1u + (uint32_t)C::kStagesPerKeyTile * (uint32_t)count_key_tiles(p, item);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           uint32_t qv[32];

@@ -724,6 +724,21 @@ rk_status rk_segmented_merge(rk_ctx* ctx, int32_t n_parts, int64_t n_rows, int32
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "merge launch");
 }
 
+rk_status rk_segmented_merge_phase(rk_ctx* ctx, const rk_request* rq, int32_t seg_begin, int32_t n_parts, int64_t n_rows,
+                                   int32_t n_heads, const void* O_part, int32_t part_dtype, const float* lse_part,
+                                   const int32_t* row_pos, void* O, float* lse, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  if (!rq || !O_part || !lse_part || !O || !lse) return fail(ctx, RK_ERR_NULL, "null argument");
+  if (rq->ctx != ctx) return fail(ctx, RK_ERR_LAYOUT, "request belongs to another context");
+  if (n_parts <= 0 || n_parts > kMergeMaxParts || n_rows < 0 || n_heads <= 0) return fail(ctx, RK_ERR_LAYOUT, "bad part/row/head count");
+  if (seg_begin < 0 || seg_begin + n_parts > rq->S) return fail(ctx, RK_ERR_LAYOUT, "segment range out of bounds");
+  if (part_dtype != 0 && part_dtype != 1) return fail(ctx, RK_ERR_UNSUPPORTED, "part_dtype must be 0 (bf16) or 1 (fp32)");
+  if (!aligned16(O_part) || !aligned16(O)) return fail(ctx, RK_ERR_ALIGN, "O_part/O must be 16-byte aligned");
+  cudaError_t e = launch_merge_phase(n_parts, n_rows, n_heads, O_part, part_dtype, lse_part, rq->d_seg_cs + (size_t)seg_begin * 32,
+                                     row_pos, ctx->rope_turns, O, lse, ctx->sm_count, reinterpret_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "merge launch");
+}
+
 static rk_status run_gemm(rk_ctx* ctx, const void* A, int64_t a_rows, int64_t a_cols, const void* B, int64_t b_rows,
                           int64_t b_cols, void* C, int64_t ldc, int M, int N, int K, int batch_off, int n_batches,
                           cudaStream_t st) {

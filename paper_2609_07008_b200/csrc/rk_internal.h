@@ -86,6 +86,9 @@ cudaError_t launch_relocate(const void* q_rope, int64_t n_rows, int32_t n_heads,
                             void* out, int sm_count, cudaStream_t stream);
 cudaError_t launch_merge(int32_t n_parts, int64_t n_rh, const void* O_part, int32_t part_dtype,
                          const float* lse_part, void* O, float* lse, int sm_count, cudaStream_t stream);
+cudaError_t launch_merge_phase(int32_t n_parts, int64_t n_rows, int32_t n_heads, const void* O_part, int32_t part_dtype,
+                               const float* lse_part, const float2* seg_cs, const int32_t* row_pos, const double* rope_turns,
+                               void* O, float* lse, int sm_count, cudaStream_t stream);
 cudaError_t launch_combine(const void* z_on_g, const void* z_on_l, const void* z_off, const int32_t* inv_map,
                            int64_t T, int64_t width, void* z, int sm_count, cudaStream_t stream);
 

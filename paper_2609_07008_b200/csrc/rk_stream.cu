@@ -127,6 +127,110 @@ __global__ void __launch_bounds__(256) rk_merge_kernel(int32_t n_parts, int64_t 
   }
 }
 
+// The merge for per-segment partial results of the output-phase variant (Algorithm 2: RestorePhase, then
+// SegmentedLSEMerge, then the inverse output RoPE of Eq. offonline).  Rows are 576 wide; the 512 latent dims
+// merge as above, the 64 rope dims (lanes 0-7, 8 dims = 4 rotation pairs each) are turned by
+// R(+delta of the part's segment) before they are added and by R(-row position) at the end.
+struct MergePhaseArgs {
+  const float2* seg_cs;    // [S][32] (cos, sin)(delta_i theta_j), first part's segment first
+  const int32_t* row_pos;  // [n_rows] or nullptr
+  int32_t n_heads;
+  double rope_turns[32];   // theta_j / (2 pi)
+};
+
+template <bool kF32>
+__global__ void __launch_bounds__(256) rk_merge_phase_kernel(int32_t n_parts, int64_t n_rh, const void* __restrict__ O_part,
+                                                             const float* __restrict__ lse_part, const MergePhaseArgs a,
+                                                             __nv_bfloat16* __restrict__ O, float* __restrict__ lse) {
+  extern __shared__ float wsm[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float* w = wsm + (size_t)warp * n_parts;
+  const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  for (int64_t rh = (int64_t)blockIdx.x * (blockDim.x >> 5) + warp; rh < n_rh; rh += n_warps) {
+    float mx = -INFINITY;
+    for (int j = lane; j < n_parts; j += 32) {
+      const float l = __ldg(lse_part + (int64_t)j * n_rh + rh);
+      w[j] = l;
+      mx = fmaxf(mx, l);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    const float m_safe = (mx == -INFINITY) ? 0.f : mx;
+    float tot = 0.f;
+    __syncwarp();
+    for (int j = lane; j < n_parts; j += 32) {
+      const float e = __expf(w[j] - m_safe);
+      w[j] = e;
+      tot += e;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+    __syncwarp();
+    const float inv = tot > 0.f ? 1.f / tot : 0.f;
+    float acc[16], accr[8];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) accr[e] = 0.f;
+    for (int j = 0; j < n_parts; ++j) {
+      const float wj = w[j] * inv;
+      if (wj > 0.f) {
+        float f[24];
+        if (kF32) {
+          const float* src = reinterpret_cast<const float*>(O_part) + ((int64_t)j * n_rh + rh) * 576;
+#pragma unroll
+          for (int hlf = 0; hlf < 2; ++hlf) {
+            const float4 x = __ldcs(reinterpret_cast<const float4*>(src + 256 * hlf + 8 * lane));
+            const float4 y = __ldcs(reinterpret_cast<const float4*>(src + 256 * hlf + 8 * lane + 4));
+            f[8 * hlf + 0] = x.x; f[8 * hlf + 1] = x.y; f[8 * hlf + 2] = x.z; f[8 * hlf + 3] = x.w;
+            f[8 * hlf + 4] = y.x; f[8 * hlf + 5] = y.y; f[8 * hlf + 6] = y.z; f[8 * hlf + 7] = y.w;
+          }
+          if (lane < 8) {
+            const float4 x = __ldcs(reinterpret_cast<const float4*>(src + 512 + 8 * lane));
+            const float4 y = __ldcs(reinterpret_cast<const float4*>(src + 512 + 8 * lane + 4));
+            f[16] = x.x; f[17] = x.y; f[18] = x.z; f[19] = x.w; f[20] = y.x; f[21] = y.y; f[22] = y.z; f[23] = y.w;
+          }
+        } else {
+          const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(O_part) + ((int64_t)j * n_rh + rh) * 576;
+          unpack8(__ldcs(reinterpret_cast<const uint4*>(src + 8 * lane)), f);
+          unpack8(__ldcs(reinterpret_cast<const uint4*>(src + 256 + 8 * lane)), f + 8);
+          if (lane < 8) unpack8(__ldcs(reinterpret_cast<const uint4*>(src + 512 + 8 * lane)), f + 16);
+        }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[e] += wj * f[e];
+        if (lane < 8) {  // RestorePhase: R(+delta): (x0, x1) -> (x0 cos - x1 sin, x0 sin + x1 cos)
+          const float4* cs = reinterpret_cast<const float4*>(a.seg_cs + (size_t)j * 32 + 4 * lane);
+          const float4 t01 = __ldg(cs), t23 = __ldg(cs + 1);
+          accr[0] += wj * (f[16] * t01.x - f[17] * t01.y);  accr[1] += wj * (f[16] * t01.y + f[17] * t01.x);
+          accr[2] += wj * (f[18] * t01.z - f[19] * t01.w);  accr[3] += wj * (f[18] * t01.w + f[19] * t01.z);
+          accr[4] += wj * (f[20] * t23.x - f[21] * t23.y);  accr[5] += wj * (f[20] * t23.y + f[21] * t23.x);
+          accr[6] += wj * (f[22] * t23.z - f[23] * t23.w);  accr[7] += wj * (f[22] * t23.w + f[23] * t23.z);
+        }
+      }
+    }
+    __nv_bfloat16* dst = O + rh * 576;
+    *reinterpret_cast<uint4*>(dst + 8 * lane) = pack8(acc);
+    *reinterpret_cast<uint4*>(dst + 256 + 8 * lane) = pack8(acc + 8);
+    if (lane < 8) {
+      if (a.row_pos != nullptr) {  // inverse output RoPE at the row's request position
+        const int pos = a.row_pos[rh / a.n_heads];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const double t = -(double)pos * a.rope_turns[4 * lane + i];
+          float sn, c;
+          sincospif(2.f * (float)(t - rint(t)), &sn, &c);
+          const float x0 = accr[2 * i], x1 = accr[2 * i + 1];
+          accr[2 * i] = x0 * c - x1 * sn;
+          accr[2 * i + 1] = x0 * sn + x1 * c;
+        }
+      }
+      *reinterpret_cast<uint4*>(dst + 512 + 8 * lane) = pack8(accr);
+    }
+    if (lane == 0) lse[rh] = tot > 0.f ? m_safe + logf(tot) : -INFINITY;
+    __syncwarp();
+  }
+}
+
 // z = z_on_g + (protected ? z_on_l[slot] : z_off[row]): a per-row select, never an add of both.
 __global__ void __launch_bounds__(256) rk_combine_kernel(const __nv_bfloat16* __restrict__ z_on_g,
                                                          const __nv_bfloat16* __restrict__ z_on_l,
@@ -165,8 +269,31 @@ inline int grid_for(int64_t n_threads_needed, int sm_count, int per_sm) {
 cudaError_t stream_setup() {
   const int bytes = 8 * kMergeMaxParts * (int)sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(rk_merge_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(rk_merge_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(rk_merge_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(rk_merge_phase_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(rk_merge_phase_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  return e;
+}
+
+cudaError_t launch_merge_phase(int32_t n_parts, int64_t n_rows, int32_t n_heads, const void* O_part, int32_t part_dtype,
+                               const float* lse_part, const float2* seg_cs, const int32_t* row_pos, const double* rope_turns,
+                               void* O, float* lse, int sm_count, cudaStream_t stream) {
+  const int64_t n_rh = n_rows * n_heads;
+  if (n_rh == 0) return cudaSuccess;
+  MergePhaseArgs a;
+  a.seg_cs = seg_cs;
+  a.row_pos = row_pos;
+  a.n_heads = n_heads;
+  for (int j = 0; j < 32; ++j) a.rope_turns[j] = rope_turns[j];
+  const size_t smem = (size_t)8 * n_parts * sizeof(float);
+  const int grid = grid_for(n_rh * 32, sm_count, 8);
+  if (part_dtype == 1)
+    rk_merge_phase_kernel<true><<<grid, 256, smem, stream>>>(n_parts, n_rh, O_part, lse_part, a,
+                                                              reinterpret_cast<__nv_bfloat16*>(O), lse);
+  else
+    rk_merge_phase_kernel<false><<<grid, 256, smem, stream>>>(n_parts, n_rh, O_part, lse_part, a,
+                                                               reinterpret_cast<__nv_bfloat16*>(O), lse);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_relocate(const void* q_rope, int64_t n_rows, int32_t n_heads, int64_t row_stride,

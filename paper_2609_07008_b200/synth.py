@@ -238,11 +238,13 @@ def _normal_big(shape, std, gen, device, chunk_rows=1 << 16):
 
 def make_tensors(name: str, profile: Profile, layout: Layout, prot_rows: np.ndarray, seed: int,
                  device="cpu", regime: str = "mandated", with_q_all: bool = False,
-                 z_off_std: float = 0.02) -> Workload:
+                 z_off_std: float = 0.02, value_phase: bool = False) -> Workload:
     """regime 'mandated': bf16 N(0, 0.02) latents and weights, q ~ N(0, 1) (the stated
     benchmark values; softmax is then close to uniform).  regime 'sharp': latents N(0, 1),
     q ~ N(0, 1.2), so that logits have a standard deviation near 2 and any masking or
-    relocation error changes the output at O(1)."""
+    relocation error changes the output at O(1).  value_phase: the output-phase variant, whose
+    value is the whole stored row: W_uv is [H, 128, 576] (everything else is drawn as before, in
+    the same order, so the other tensors of a seed do not depend on the flag up to W_uv)."""
     dev = torch.device(device)
     gen = torch.Generator(device=dev)
     gen.manual_seed(int(seed) * 7919 + (0 if regime == "mandated" else 1))
@@ -262,7 +264,7 @@ def make_tensors(name: str, profile: Profile, layout: Layout, prot_rows: np.ndar
     else:
         q_g = _normal_big((T, G, dqk), q_std, gen, dev)
         q_l = _normal_big((A, L, dqk), q_std, gen, dev)
-    w_uv = _normal((H, profile.d_v, profile.d_latent), 0.02, gen, dev)
+    w_uv = _normal((H, profile.d_v, profile.d_qk if value_phase else profile.d_latent), 0.02, gen, dev)
     w_a = _normal((G, profile.o_rank, GROUP_SIZE * profile.d_v), 0.02, gen, dev)
     w_b = _normal((profile.d_model, G * profile.o_rank), 0.02, gen, dev)
     z_off = _normal_big((layout.n_doc_rows, G * profile.o_rank), z_off_std, gen, dev)
@@ -271,17 +273,17 @@ def make_tensors(name: str, profile: Profile, layout: Layout, prot_rows: np.ndar
 
 
 def make_workload(name: str, device="cpu", regime: str = "mandated", layer: int = 0,
-                  with_q_all: bool = False, seed: Optional[int] = None) -> Workload:
+                  with_q_all: bool = False, seed: Optional[int] = None, value_phase: bool = False) -> Workload:
     profile, layout, prot = make_geometry(name, layer=layer, seed=seed)
     base_seed = CONFIGS[name]["seed"] if seed is None else seed
     return make_tensors(name, profile, layout, prot, base_seed * 1000 + layer, device=device,
-                        regime=regime, with_q_all=with_q_all)
+                        regime=regime, with_q_all=with_q_all, value_phase=value_phase)
 
 
 def make_custom(doc_lens: Sequence[int], n_query: int, n_heads: int, n_groups: int, o_rank: int,
                 d_model: int, pct_bp: int, seed: int, device="cpu", regime: str = "sharp",
                 shuffle: bool = True, run_len: int = 1, with_q_all: bool = False,
-                base_delta: int = 0) -> Workload:
+                base_delta: int = 0, value_phase: bool = False) -> Workload:
     """Free-form small case for parity tests (ragged lengths, odd sizes)."""
     rng = np.random.default_rng(np.random.PCG64(seed))
     layout = make_layout(doc_lens, n_query, rng, shuffle, base_delta=base_delta)
@@ -290,7 +292,7 @@ def make_custom(doc_lens: Sequence[int], n_query: int, n_heads: int, n_groups: i
     profile = Profile(n_heads=n_heads, n_groups=n_groups, o_rank=o_rank, d_model=d_model,
                       global_heads=gh, sm_scale=float(1.0 / np.sqrt(D_V + D_ROPE)))
     return make_tensors("custom", profile, layout, prot, seed, device=device, regime=regime,
-                        with_q_all=with_q_all)
+                        with_q_all=with_q_all, value_phase=value_phase)
 
 
 def sample_rows(layout: Layout, prot_rows: np.ndarray, n_random: int, seed: int,
@@ -368,7 +370,7 @@ def draw_router_weights(n: int, seed: int, temperature: float = 1.5, tie_share: 
 
 
 def make_random_request(seed: int, n_heads: int = 16, n_groups: int = 2, o_rank: int = 256, d_model: int = 512,
-                        regime: str = "sharp", device="cpu") -> Workload:
+                        regime: str = "sharp", device="cpu", value_phase: bool = False) -> Workload:
     """A seeded irregular request for edge-case parity: 2-7 segments whose lengths mix tile-boundary
     values (1, 2, 63..65, 127..129, 255..257) with random ones, a random request order with random gaps
     between segments, some segments in the middle without artifact (new rows), a short query suffix
@@ -396,4 +398,4 @@ def make_random_request(seed: int, n_heads: int = 16, n_groups: int = 2, o_rank:
     prot = draw_protected_rows(layout, int(rng.integers(0, 3000)), rng)
     profile = Profile(n_heads=n_heads, n_groups=n_groups, o_rank=o_rank, d_model=d_model,
                       global_heads=draw_global_heads(n_groups, rng), sm_scale=float(1.0 / np.sqrt(D_V + D_ROPE)))
-    return make_tensors("random", profile, layout, prot, seed, device=device, regime=regime)
+    return make_tensors("random", profile, layout, prot, seed, device=device, regime=regime, value_phase=value_phase)
