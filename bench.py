@@ -84,11 +84,80 @@ class ClockSampler(threading.Thread):
                     samples=len(self.samples))
 
 
-def algorithmic_flops(profile, req):
-    """Work the method itself must do: Global heads x all rows + Local heads x protected rows."""
+class NvmlClock(threading.Thread):
+    """SM clock of one GPU read through NVML every few milliseconds (nvidia-smi is too slow for a region of a
+    few hundred milliseconds).  Read-only: nothing is set."""
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        super().__init__(daemon=True)
+        self.index, self.period, self.samples, self.stop_flag, self.ok = index, period_s, [], False, False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.max_mhz = None
+
+    def run(self):
+        while self.ok and not self.stop_flag:
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def median(self):
+        v = sorted(self.samples)
+        return v[len(v) // 2] if v else None
+
+
+def timed_region(fn, stream, gpu_index, min_ms=300.0, lead_ms=30.0):
+    """Times one call `fn` in its steady state: the same call is first repeated for at least lead_ms, then
+    timed back to back (CUDA events on the launching stream) over at least 20 repeats and min_ms, with the
+    SM clock sampled through NVML during the timed repeats.  Returns (ms per call, median SM MHz, max SM MHz)."""
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    fn()
+    b.record(stream)
+    torch.cuda.synchronize()
+    one = max(a.elapsed_time(b), 1e-3)
+    for _ in range(max(3, int(lead_ms / one))):
+        fn()
+    reps = max(20, int(min_ms / one))
+    clk = NvmlClock(gpu_index)
+    torch.cuda.synchronize()
+    clk.start()
+    a.record(stream)
+    for _ in range(reps):
+        fn()
+    b.record(stream)
+    torch.cuda.synchronize()
+    clk.stop_flag = True
+    clk.join(timeout=1)
+    return a.elapsed_time(b) / reps, clk.median(), clk.max_mhz
+
+
+def hbm_entry(ms, nbytes, mhz, max_mhz, **kw):
+    """One standalone HBM-bound kernel: GB/s as measured, the SM clock it ran at, and GB/s scaled to the maximum
+    clock (what an issue- or latency-bound kernel would read at full clock; a DRAM-bound one does not scale)."""
+    gbs = nbytes / ms / 1e6
+    d = dict(ms=ms, bytes=nbytes, gbs=gbs, sm_mhz=mhz, sm_max_mhz=max_mhz, **kw)
+    if mhz and max_mhz:
+        d["gbs_at_max_clock"] = gbs * max_mhz / mhz
+    return d
+
+
+def algorithmic_flops(profile, req, value_phase=False):
+    """Work the method itself must do: Global heads x all rows + Local heads x protected rows.  In the
+    output-phase variant the value is the whole 576-wide row: 2*576 + 2*576 flop per visible pair and a
+    576-wide W_uv."""
     G, L, ro, dm = profile.n_groups, profile.n_local, profile.o_rank, profile.d_model
-    attn = FLOP_PER_PAIR * (G * req.pairs_global + L * req.pairs_local)
-    proj = 2 * req.T * G * (512 * 128 + 128 * ro) + 2 * req.A * (L * 512 * 128 + G * 7 * 128 * ro)
+    ow = 576 if value_phase else 512
+    attn = (2 * 576 + 2 * ow) * (G * req.pairs_global + L * req.pairs_local)
+    proj = 2 * req.T * G * (ow * 128 + 128 * ro) + 2 * req.A * (L * ow * 128 + G * 7 * 128 * ro)
     wb = 2 * req.T * G * ro * dm
     return attn, proj, wb
 
@@ -97,7 +166,7 @@ def algorithmic_flops(profile, req):
 # CPU checker timing (cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------
 
-def oracle_sample_run(w, rows):
+def oracle_sample_run(w, rows, value_phase=False):
     """Runs the float64 checker on the packed rows `rows`; returns (seconds, visible pairs)."""
     import oracle
     from oracle.harness import f64
@@ -114,8 +183,9 @@ def oracle_sample_run(w, rows):
     vis = np.searchsorted(srt, pos[rows], side="right")
     pairs = int(sum(v * (p.n_heads if inv[r] >= 0 else p.n_groups) for v, r in zip(vis, rows)))
     t0 = time.perf_counter()
-    out = oracle.mla_online_rows(rows, q_g_rows, ql, kv, lay.seg_off, lay.seg_delta, w.prot_rows, p.global_heads,
-                                 p.local_heads, wuv, wa, wb, zo, p.sm_scale, p.rope_base, p.d_latent)
+    fn = oracle.phase.mla_online_rows_phase if value_phase else oracle.mla_online_rows
+    out = fn(rows, q_g_rows, ql, kv, lay.seg_off, lay.seg_delta, w.prot_rows, p.global_heads,
+             p.local_heads, wuv, wa, wb, zo, p.sm_scale, p.rope_base, p.d_latent)
     dt = time.perf_counter() - t0
     return dt, pairs, out
 
@@ -153,7 +223,8 @@ def run_reference(args, rank, world):
         return
     name = args.config
     prof, lay, prot = synth.make_geometry(name)
-    w = synth.make_tensors(name, prof, lay, prot, synth.CONFIGS[name]["seed"] * 1000, device="cpu")
+    w = synth.make_tensors(name, prof, lay, prot, synth.CONFIGS[name]["seed"] * 1000, device="cpu",
+                           value_phase=args.value_phase)
     import oracle
     pos = oracle.request_positions(lay.seg_off, lay.seg_delta)
     srt = np.sort(pos)
@@ -164,7 +235,7 @@ def run_reference(args, rank, world):
     rows = pick_oracle_rows(w, max(1, args.oracle_pairs // 3))
     times, pairs = [], 0
     for i in range(args.warmup + args.steps):
-        dt, pairs, _ = oracle_sample_run(w, rows)
+        dt, pairs, _ = oracle_sample_run(w, rows, args.value_phase)
         if i >= args.warmup:
             times.append(dt)
     sec = float(np.mean(times))
@@ -173,7 +244,7 @@ def run_reference(args, rank, world):
     line = dict(metric="mla_online_prefill_tokens_per_s_per_layer", value=tok_s, unit="tokens/s", n_gpus=world,
                 steps=args.steps, warmup=args.warmup, ms_per_step=sec * 1e3 * all_pairs / pairs,
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                impl="reference", config=dict(workload=name, T=lay.n_rows, n_prot=len(prot)),
+                impl="reference", config=dict(workload=name, T=lay.n_rows, n_prot=len(prot), value_phase=args.value_phase),
                 cpu_baseline=dict(value=tok_s, unit="tokens/s", cores=cores, kind="oracle",
                                   sample=f"{len(rows)} seeded rows, {pairs} of {all_pairs} visible (row,key,head) "
                                          f"pairs per step, extrapolated by pair count"),
@@ -185,30 +256,20 @@ def run_reference(args, rank, world):
 
 def time_stream_kernels(ctx, req, w, prof, lay, dev, budget_bytes=6 << 30):
     """rk_relocate_q over (rows x Global heads x frames) and rk_segmented_merge over
-    (query-suffix rows x all heads x parts), each sized to a few GB, timed with CUDA events
-    after three warm-ups; algorithmic bytes = every tensor read or written once."""
+    (query-suffix rows x all heads x parts), each sized to a few GB (far beyond L2), timed in their steady
+    state (see timed_region); algorithmic bytes = every tensor read or written once."""
     res = {}
     stream = torch.cuda.current_stream()
-
-    def timed(fn, reps=5):
-        for _ in range(3):
-            fn()
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
-        for a, b in evs:
-            a.record(stream)
-            fn()
-            b.record(stream)
-        torch.cuda.synchronize()
-        return float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    gpu = dev.index or 0
 
     G, S, T = prof.n_groups, lay.n_segs, lay.n_rows
     frame_bytes = T * G * 64 * 2
     frames = int(max(1, min(S, budget_bytes // frame_bytes)))
     out = torch.empty((frames, T, G, 64), dtype=torch.bfloat16, device=dev)
     view = w.q_g[:, :, 512:]
-    ms = timed(lambda: ctx.rk_relocate_q(req, view, 0, frames, out))
+    ms, mhz, mx = timed_region(lambda: ctx.rk_relocate_q(req, view, 0, frames, out), stream, gpu)
     nbytes = frame_bytes * (1 + frames)
-    res["rk_relocate_q"] = dict(ms=ms, bytes=nbytes, gbs=nbytes / ms / 1e6, frames=frames, rows=T, heads=G)
+    res["rk_relocate_q"] = hbm_entry(ms, nbytes, mhz, mx, frames=frames, rows=T, heads=G)
     del out
     H = prof.n_heads
     n_q = int(lay.seg_off[-1] - lay.seg_off[-2])
@@ -218,9 +279,9 @@ def time_stream_kernels(ctx, req, w, prof, lay, dev, budget_bytes=6 << 30):
     lse_part = torch.randn((parts, n_q, H), device=dev, dtype=torch.float32)
     O = torch.empty((n_q, H, 512), dtype=torch.bfloat16, device=dev)
     lse = torch.empty((n_q, H), dtype=torch.float32, device=dev)
-    ms = timed(lambda: ctx.rk_segmented_merge(O_part, lse_part, O, lse))
+    ms, mhz, mx = timed_region(lambda: ctx.rk_segmented_merge(O_part, lse_part, O, lse), stream, gpu)
     nbytes = part_bytes * parts + n_q * H * (512 * 2 + 4)
-    res["rk_segmented_merge"] = dict(ms=ms, bytes=nbytes, gbs=nbytes / ms / 1e6, parts=parts, rows=n_q, heads=H)
+    res["rk_segmented_merge"] = hbm_entry(ms, nbytes, mhz, mx, parts=parts, rows=n_q, heads=H)
     ctx.rk_poll_status()
     return res
 
@@ -231,17 +292,7 @@ def time_selection_rules(ctx, lay, dev):
     rk_moe_fanout on 16 M tokens (26 B per token, a plain streaming pass)."""
     from paper_2609_07008_b200 import synth as _synth
     stream = torch.cuda.current_stream()
-
-    def timed(fn, reps=10):
-        for _ in range(3):
-            fn()
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
-        for a, b in evs:
-            a.record(stream)
-            fn()
-            b.record(stream)
-        torch.cuda.synchronize()
-        return float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    gpu = dev.index or 0
 
     res = {}
     dirty, scores = _synth.draw_policy_inputs(lay, seed=99, n_dirty=500)
@@ -249,19 +300,20 @@ def time_selection_rules(ctx, lay, dev):
     T, S = lay.n_rows, lay.n_segs
     out = ctx.rk_protected_rows(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, d, s, budget_bp=2500)
     ws = torch.empty(16 << 20, dtype=torch.uint8, device=dev)
-    ms = timed(lambda: ctx.rk_protected_rows(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, d, s, budget_bp=2500,
-                                             out=out, workspace=ws))
+    ms, mhz, mx = timed_region(lambda: ctx.rk_protected_rows(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, d, s,
+                                                             budget_bp=2500, out=out, workspace=ws), stream, gpu, min_ms=100.0)
     n_sel = int(out[1].item())
     # per row: flag pass 1 B written; 8 select passes 1 B flag + 4 B score; count 5 B; scatter 5 B + output
     nbytes = T * (1 + 8 * 5 + 5 + 5) + 4 * n_sel + 4 * len(dirty)
     res["rk_protected_rows"] = dict(ms=ms, rows=T, selected=n_sel, budget_bp=2500, launches=13, bytes=nbytes,
-                                    gbs=nbytes / ms / 1e6, bound="launch latency (13 short kernels + 4 small copies)")
-    n = 16 << 20
+                                    gbs=nbytes / ms / 1e6, sm_mhz=mhz,
+                                    bound="launch latency (13 short kernels + 4 small copies)")
+    n = 64 << 20                           # 1.6 GB of router weights: far beyond L2
     p = torch.rand((n, 6), device=dev, dtype=torch.float32) + 0.01
     k, keep = ctx.rk_moe_fanout(p, 0.85)
-    ms = timed(lambda: ctx.rk_moe_fanout(p, 0.85, False, k, keep))
+    ms, mhz, mx = timed_region(lambda: ctx.rk_moe_fanout(p, 0.85, False, k, keep), stream, gpu)
     nbytes = n * 26
-    res["rk_moe_fanout"] = dict(ms=ms, tokens=n, bytes=nbytes, gbs=nbytes / ms / 1e6)
+    res["rk_moe_fanout"] = hbm_entry(ms, nbytes, mhz, mx, tokens=n)
     ctx.rk_poll_status()
     return res
 
@@ -320,6 +372,9 @@ def main():
     ap.add_argument("--protect-bp", type=int, default=None,
                     help="override the share of protected document rows (basis points), e.g. the paper's controller "
                          "budgets 1000 / 2000 / 2500; default: the configuration's own share")
+    ap.add_argument("--value-phase", action="store_true",
+                    help="the output-phase variant: the whole stored row is the value (RestorePhase per segment and "
+                         "the inverse output RoPE inside the attention kernel), W_uv 576 wide")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-aux", action="store_true", help="skip the standalone relocation / merge timings")
     ap.add_argument("--with-offline", action="store_true", help="also time the offline artifact build")
@@ -354,9 +409,9 @@ def main():
         prof, lay, prot = synth.make_geometry(name, layer=l, pct_bp=args.protect_bp)
         # every rank gets its own request values (independent requests, same shape)
         wl = synth.make_tensors(name, prof, lay, prot, rkdist.rank_seed(synth.CONFIGS[name]["seed"], rank) + 7 * l,
-                                device=dev, regime=args.regime)
+                                device=dev, regime=args.regime, value_phase=args.value_phase)
         if ctx is None:
-            ctx = rk.Context.from_profile(prof)
+            ctx = rk.Context.from_profile(prof, value_phase=args.value_phase)
         layers.append((wl, ctx.rk_request_create(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, prot)))
     w, req = layers[0]
     prof, lay = w.profile, w.layout
@@ -364,7 +419,7 @@ def main():
     bufs = ctx.alloc_layer_buffers(big, dev)          # staging/outputs shared by the layers (they run in sequence)
     fl_attn = fl_proj = fl_wb = 0
     for _, r in layers:
-        a, b, c = algorithmic_flops(prof, r)
+        a, b, c = algorithmic_flops(prof, r, args.value_phase)
         fl_attn, fl_proj, fl_wb = fl_attn + a, fl_proj + b, fl_wb + c
     in_bytes = sum(t.numel() * t.element_size() for wl, _ in layers for t in (wl.kv, wl.q_g, wl.q_l, wl.z_off))
     need_flush = in_bytes < 4 * L2_BYTES
@@ -455,21 +510,15 @@ def main():
 
     # standalone HBM-bound calls (not part of the step): relocation and merge against copy bandwidth
     aux = None
-    if not args.no_aux and rank == 0:
+    if not args.no_aux and rank == 0 and not args.value_phase:
         aux = time_stream_kernels(ctx, req, w, prof, lay, dev)
         aux.update(time_selection_rules(ctx, lay, dev))
 
     # where the rest of the step goes (instrumentation pass, not the timed region)
     breakdown = None
     if rank == 0:
-        def ev_ms(fn, reps=3):
-            fn()
-            out = []
-            for _ in range(reps):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream); fn(); b.record(stream); torch.cuda.synchronize()
-                out.append(a.elapsed_time(b))
-            return float(np.mean(out))
+        def ev_ms(fn):
+            return timed_region(fn, stream, dev.index or 0, min_ms=150.0, lead_ms=20.0)[0]
         t_proj = ev_ms(lambda: ctx.rk_group_sliced_proj(req, bufs["O_g"], bufs["O_l"], w.w_uv, w.w_a, bufs["z_on_g"],
                                                         bufs["z_on_l"], bufs["workspace"]))
         t_comb = ev_ms(lambda: ctx.rk_combine_offline(req, bufs["z_on_g"], bufs["z_on_l"], w.z_off, None, bufs["z"]))
@@ -493,13 +542,14 @@ def main():
 
     peaks = load_peaks()
     attn_tflops = fl_attn / (np.mean(attn_ms) * 1e-3) / 1e12
-    roofline = dict(bound="tensor", kernel="rk_mla_attn_kernel (Global + Local launches)",
+    roofline = dict(bound="tensor", kernel="rk_mla_attn_kernel (Global + Local launches)" +
+                                           (", output-phase instantiation, 2304 flop per pair" if args.value_phase else ""),
                     achieved=attn_tflops, peak=peaks["bf16_sustained"], unit="TFLOP/s",
                     frac=attn_tflops / peaks["bf16_sustained"], peak_source=peaks["source"] + " sustained bf16",
                     frac_of_burst=attn_tflops / peaks["bf16_burst"], frac_of_nominal=attn_tflops / 2250.0,
                     launches_per_step=2 * n_layers, ms_per_step=float(np.mean(attn_ms)),
                     ms_global_pass=float(np.mean(attn_g_ms)),
-                    traffic=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("bytes"),
+                    traffic=None if args.value_phase else (PROFILED_DRAM_TRAFFIC.get(name) or {}).get("bytes"),
                     traffic_note=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("source", "no ncu capture of this workload"),
                     algorithmic_dram_bytes=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("algorithmic"))
     rest_tflops = (fl_proj + fl_wb) / (np.mean(rest_ms) * 1e-3) / 1e12
@@ -509,7 +559,7 @@ def main():
         run_layer(w, req)                      # leave layer 0's y in the buffer for the parity figure below
         torch.cuda.synchronize()
         rows = pick_oracle_rows(w, args.oracle_pairs)
-        dt, pairs, out = oracle_sample_run(w, rows)
+        dt, pairs, out = oracle_sample_run(w, rows, args.value_phase)
         allp = total_pairs(prof, req)          # layer 0 (the layers have the same layout, own protected rows)
         # while the sample is at hand: parity of this very run against the checker
         from oracle.harness import rel_l2
@@ -525,7 +575,7 @@ def main():
                 unit="tokens/s", n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=total_ms_max / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="bf16", data="synthetic",
-                config=dict(workload=name, regime=args.regime, layers=n_layers, T=req.T, n_prot=req.A, n_segs=lay.n_segs,
+                config=dict(workload=name, regime=args.regime, value_phase=args.value_phase, layers=n_layers, T=req.T, n_prot=req.A, n_segs=lay.n_segs,
                             heads=prof.n_heads, groups=prof.n_groups, o_rank=prof.o_rank, d_model=prof.d_model,
                             l2="inputs larger than L2" if not need_flush else "L2 flushed between iterations",
                             flops_attn=fl_attn, flops_proj=fl_proj + fl_wb),

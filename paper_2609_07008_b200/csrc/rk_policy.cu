@@ -204,19 +204,12 @@ __global__ void __launch_bounds__(kPolicyThreads) policy_scatter_kernel(PolicyPa
   if (sel) p.rows_out[p.block_counts[blockIdx.x] + warp_sums[warp] + __popc(ballot & ((1u << lane) - 1u))] = t;
 }
 
-// Eq. (moe): one token per thread.  The six weights are sorted by a 12-exchange min/max network
-// (values only: equal weights are interchangeable in the sums); which slots stay follows from each
-// slot's rank, counted pairwise with the tie rule "lower slot first".
-__global__ void __launch_bounds__(256) moe_fanout_kernel(const float* __restrict__ p, long long n, float tau, int fence,
-                                                         uint8_t* __restrict__ k_out, uint8_t* __restrict__ keep_out) {
-  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= n) return;
-  // 24 bytes per thread as three 8-byte loads: staging a warp's 768 bytes through shared memory for
-  // fully coalesced loads was measured slower (the kernel is as much issue-bound as memory-bound)
-  const float2* src = reinterpret_cast<const float2*>(p + 6 * t);
-  const float2 a = __ldcs(src), b = __ldcs(src + 1), c = __ldcs(src + 2);
-  const float w[6] = {a.x, a.y, b.x, b.y, c.x, c.y};
-  float s[6] = {a.x, a.y, b.x, b.y, c.x, c.y};
+// Eq. (moe) for one token.  The six weights are sorted by a 12-exchange min/max network (values only:
+// equal weights are interchangeable in the sums); the sums run in sorted order in float32.  Which slots
+// stay: every slot above the K_t-th largest value, and of the slots equal to it as many of the lowest as
+// are still needed (equal weights: lower slot first).  Returns K_t | keep << 8.
+__device__ __forceinline__ unsigned moe_fanout_token(const float (&w)[6], float tau, int fence) {
+  float s[6] = {w[0], w[1], w[2], w[3], w[4], w[5]};
 #define RK_CE(i, j) { const float hi = fmaxf(s[i], s[j]), lo = fminf(s[i], s[j]); s[i] = hi; s[j] = lo; }
   RK_CE(0, 5) RK_CE(1, 3) RK_CE(2, 4)
   RK_CE(1, 2) RK_CE(3, 4)
@@ -224,32 +217,74 @@ __global__ void __launch_bounds__(256) moe_fanout_kernel(const float* __restrict
   RK_CE(0, 1) RK_CE(2, 3) RK_CE(4, 5)
   RK_CE(1, 2) RK_CE(3, 4)
 #undef RK_CE
-  float cum = __fadd_rn(__fadd_rn(s[0], s[1]), s[2]);
-  const float c3 = cum;
+  const float c3 = __fadd_rn(__fadd_rn(s[0], s[1]), s[2]);
   const float c4 = __fadd_rn(c3, s[3]);
   const float c5 = __fadd_rn(c4, s[4]);
   const float c6 = __fadd_rn(c5, s[5]);
   int k = 6;
+  float v = s[5];  // the K_t-th largest value
   if (!fence) {
     const float thr = __fmul_rn(tau, c6);
-    if (c3 >= thr) k = 3;
-    else if (c4 >= thr) k = 4;
-    else if (c5 >= thr) k = 5;
+    if (c3 >= thr) { k = 3; v = s[2]; }
+    else if (c4 >= thr) { k = 4; v = s[3]; }
+    else if (c5 >= thr) { k = 5; v = s[4]; }
   }
-  int rank[6] = {0, 0, 0, 0, 0, 0};
+  unsigned gt = 0u, eq = 0u;
 #pragma unroll
-  for (int o = 0; o < 6; ++o)
-#pragma unroll
-    for (int q = o + 1; q < 6; ++q) {
-      const bool o_first = w[o] >= w[q];  // equal weights: the lower slot ranks first
-      rank[q] += o_first ? 1 : 0;
-      rank[o] += o_first ? 0 : 1;
+  for (int q = 0; q < 6; ++q) {
+    gt |= (w[q] > v ? 1u : 0u) << q;
+    eq |= (w[q] == v ? 1u : 0u) << q;
+  }
+  int need = k - __popc(gt);       // slots still to take among those equal to v (at least one)
+  unsigned keep = gt | eq;
+  if (__popc(eq) != need) {        // more equal slots than places: the lowest slots win
+    keep = gt;
+    for (unsigned m = eq; need > 0; --need) {
+      const unsigned low = m & (0u - m);
+      keep |= low;
+      m ^= low;
     }
-  unsigned keep = 0u;
+  }
+  return (unsigned)k | (keep << 8);
+}
+
+// One token per thread (any alignment; also the tail of the four-token kernel).
+__global__ void __launch_bounds__(256) moe_fanout_kernel(const float* __restrict__ p, long long n, float tau, int fence,
+                                                         uint8_t* __restrict__ k_out, uint8_t* __restrict__ keep_out) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n) return;
+  const float2* src = reinterpret_cast<const float2*>(p + 6 * t);
+  const float2 a = __ldcs(src), b = __ldcs(src + 1), c = __ldcs(src + 2);
+  const float w[6] = {a.x, a.y, b.x, b.y, c.x, c.y};
+  const unsigned r = moe_fanout_token(w, tau, fence);
+  k_out[t] = (uint8_t)(r & 0xffu);
+  keep_out[t] = (uint8_t)(r >> 8);
+}
+
+// Four consecutive tokens per thread: 96 contiguous bytes in as six 16-byte loads, the four K_t and the
+// four masks out as one 32-bit store each.  Against one token per thread that removes most of the load,
+// store and address instructions (about a tenth of the work per token) and gives every thread four
+// independent chains, which is what an issue-bound streaming kernel needs.  n4 = number of token quads.
+__global__ void __launch_bounds__(256) moe_fanout4_kernel(const float4* __restrict__ p, long long n4, float tau, int fence,
+                                                          uint32_t* __restrict__ k_out, uint32_t* __restrict__ keep_out) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n4) return;
+  const float4* src = p + 6 * t;
+  float4 v[6];
 #pragma unroll
-  for (int q = 0; q < 6; ++q) keep |= (rank[q] < k ? 1u : 0u) << q;
-  k_out[t] = (uint8_t)k;
-  keep_out[t] = (uint8_t)keep;
+  for (int i = 0; i < 6; ++i) v[i] = __ldcs(src + i);
+  const float f[24] = {v[0].x, v[0].y, v[0].z, v[0].w, v[1].x, v[1].y, v[1].z, v[1].w, v[2].x, v[2].y, v[2].z, v[2].w,
+                       v[3].x, v[3].y, v[3].z, v[3].w, v[4].x, v[4].y, v[4].z, v[4].w, v[5].x, v[5].y, v[5].z, v[5].w};
+  uint32_t kk = 0u, mm = 0u;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const float w[6] = {f[6 * u], f[6 * u + 1], f[6 * u + 2], f[6 * u + 3], f[6 * u + 4], f[6 * u + 5]};
+    const unsigned r = moe_fanout_token(w, tau, fence);
+    kk |= (r & 0xffu) << (8 * u);
+    mm |= (r >> 8) << (8 * u);
+  }
+  __stcs(k_out + t, kk);
+  __stcs(keep_out + t, mm);
 }
 
 }  // namespace
@@ -314,8 +349,23 @@ int protected_rows_launches(bool with_scores, bool with_dirty) { return 4 + (wit
 cudaError_t launch_moe_fanout(const float* p, int64_t n, float tau, int fence, uint8_t* k_out, uint8_t* keep_out,
                               cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
-  const int64_t nb = (n + 255) / 256;
-  moe_fanout_kernel<<<(unsigned)nb, 256, 0, stream>>>(p, (long long)n, tau, fence, k_out, keep_out);
+  int64_t done = 0;
+  const bool vec = (reinterpret_cast<uintptr_t>(p) & 15u) == 0 && (reinterpret_cast<uintptr_t>(k_out) & 3u) == 0 &&
+                   (reinterpret_cast<uintptr_t>(keep_out) & 3u) == 0;
+  if (vec && n >= 4) {
+    const int64_t n4 = n / 4;
+    moe_fanout4_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, stream>>>(reinterpret_cast<const float4*>(p), (long long)n4, tau,
+                                                                         fence, reinterpret_cast<uint32_t*>(k_out),
+                                                                         reinterpret_cast<uint32_t*>(keep_out));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    done = 4 * n4;
+  }
+  if (done < n) {
+    const int64_t rest = n - done;
+    moe_fanout_kernel<<<(unsigned)((rest + 255) / 256), 256, 0, stream>>>(p + 6 * done, (long long)rest, tau, fence,
+                                                                          k_out + done, keep_out + done);
+  }
   return cudaGetLastError();
 }
 

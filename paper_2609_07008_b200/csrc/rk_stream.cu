@@ -23,38 +23,52 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
   return make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
 }
 
-// One thread per 16-byte chunk (4 rotation pairs) of one (row, head); the input is read once
-// and one rotated copy is written per segment frame.
+// A thread owns kRelU 16-byte chunks (4 rotation pairs each) of the input, 256 chunks apart, so all of them
+// use the same four (cos, sin) pairs of a frame; it keeps them unpacked in registers and writes one rotated
+// copy per segment frame.  Per 16 bytes written that leaves the arithmetic, one pack and one store; the
+// kRelU independent stores per frame keep enough bytes in flight at any SM clock.
+constexpr int kRelU = 4;
 __global__ void __launch_bounds__(256) rk_relocate_kernel(const __nv_bfloat16* __restrict__ q, int64_t n_rows,
                                                           int32_t n_heads, int64_t row_stride, int64_t head_stride,
                                                           const float2* __restrict__ seg_cs, int32_t seg_begin,
                                                           int32_t n_frames, __nv_bfloat16* __restrict__ out) {
   const int64_t n_items = n_rows * n_heads * 8;
   const int64_t frame_elems = n_rows * n_heads * 64;
-  for (int64_t it = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; it < n_items;
-       it += (int64_t)gridDim.x * blockDim.x) {
-    const int c = (int)(it & 7);
-    const int64_t rh = it >> 3;
-    const int64_t r = (rh < (int64_t)0x7fffffff) ? (int64_t)((uint32_t)rh / (uint32_t)n_heads) : rh / n_heads;
-    const int h = (int)(rh - r * n_heads);
-    const uint4 v = *reinterpret_cast<const uint4*>(q + r * row_stride + h * head_stride + c * 8);
-    float x[8];
-    unpack8(v, x);
-    __nv_bfloat16* dst = out + it * 8;
+  const int c = (int)(threadIdx.x & 7);
+  const int64_t n_groups = (n_items + 256 * kRelU - 1) / (256 * kRelU);
+  for (int64_t grp = blockIdx.x; grp < n_groups; grp += gridDim.x) {
+    const int64_t it0 = grp * (256 * kRelU) + threadIdx.x;
+    float x[kRelU][8];
+#pragma unroll
+    for (int u = 0; u < kRelU; ++u) {
+      const int64_t it = it0 + u * 256;
+      if (it < n_items) {
+        const int64_t rh = it >> 3;
+        const int64_t r = (rh < (int64_t)0x7fffffff) ? (int64_t)((uint32_t)rh / (uint32_t)n_heads) : rh / n_heads;
+        const int h = (int)(rh - r * n_heads);
+        unpack8(__ldcs(reinterpret_cast<const uint4*>(q + r * row_stride + h * head_stride + c * 8)), x[u]);
+      }
+    }
     // Frames are whole multiples of a megabyte apart, so writing frame i from every block at the same
-    // time would hit the same memory channels; each block starts at a different frame instead.
-    int i = (int)(blockIdx.x % (unsigned)n_frames);
-#pragma unroll 4
+    // time would hit the same memory channels; each group of chunks starts at a different frame instead.
+    int i = (int)(grp % (int64_t)n_frames);
+#pragma unroll 2
     for (int n = 0; n < n_frames; ++n) {
       const float4* cs = reinterpret_cast<const float4*>(seg_cs + (size_t)(seg_begin + i) * 32 + 4 * c);
       const float4 t01 = __ldg(cs), t23 = __ldg(cs + 1);
-      float y[8];
-      // R(-delta): (x0, x1) -> (x0 cos + x1 sin, x1 cos - x0 sin)
-      y[0] = x[0] * t01.x + x[1] * t01.y;  y[1] = x[1] * t01.x - x[0] * t01.y;
-      y[2] = x[2] * t01.z + x[3] * t01.w;  y[3] = x[3] * t01.z - x[2] * t01.w;
-      y[4] = x[4] * t23.x + x[5] * t23.y;  y[5] = x[5] * t23.x - x[4] * t23.y;
-      y[6] = x[6] * t23.z + x[7] * t23.w;  y[7] = x[7] * t23.z - x[6] * t23.w;
-      __stcs(reinterpret_cast<uint4*>(dst + (int64_t)i * frame_elems), pack8(y));
+      __nv_bfloat16* dst = out + (int64_t)i * frame_elems + it0 * 8;
+#pragma unroll
+      for (int u = 0; u < kRelU; ++u) {
+        if (it0 + u * 256 < n_items) {
+          float y[8];
+          // R(-delta): (x0, x1) -> (x0 cos + x1 sin, x1 cos - x0 sin)
+          y[0] = x[u][0] * t01.x + x[u][1] * t01.y;  y[1] = x[u][1] * t01.x - x[u][0] * t01.y;
+          y[2] = x[u][2] * t01.z + x[u][3] * t01.w;  y[3] = x[u][3] * t01.z - x[u][2] * t01.w;
+          y[4] = x[u][4] * t23.x + x[u][5] * t23.y;  y[5] = x[u][5] * t23.x - x[u][4] * t23.y;
+          y[6] = x[u][6] * t23.z + x[u][7] * t23.w;  y[7] = x[u][7] * t23.z - x[u][6] * t23.w;
+          __stcs(reinterpret_cast<uint4*>(dst + u * 2048), pack8(y));
+        }
+      }
       i = (i + 1 == n_frames) ? 0 : i + 1;
     }
   }
@@ -94,29 +108,53 @@ __global__ void __launch_bounds__(256) rk_merge_kernel(int32_t n_parts, int64_t 
     float acc[16];
 #pragma unroll
     for (int e = 0; e < 16; ++e) acc[e] = 0.f;
-    for (int j = 0; j < n_parts; ++j) {
-      const float wj = w[j] * inv;
-      if (wj > 0.f) {
-        if (kF32) {
-          const float* src = reinterpret_cast<const float*>(O_part) + ((int64_t)j * n_rh + rh) * 512;
+    // The loads of kMergeU parts are issued together and without looking at the weights (an empty part's
+    // rows are valid memory; what they hold is never used), so that a warp keeps kMergeU KB in flight
+    // instead of one; only the arithmetic is skipped for a part of weight zero.
+    constexpr int kMergeU = 4;
+    const int64_t part_stride = n_rh * 512;
+    for (int j0 = 0; j0 < n_parts; j0 += kMergeU) {
+      float wj[kMergeU];
 #pragma unroll
-          for (int hlf = 0; hlf < 2; ++hlf) {
-            const float4 a = __ldcs(reinterpret_cast<const float4*>(src + 256 * hlf + 8 * lane));
-            const float4 b = __ldcs(reinterpret_cast<const float4*>(src + 256 * hlf + 8 * lane + 4));
-            acc[8 * hlf + 0] += wj * a.x; acc[8 * hlf + 1] += wj * a.y; acc[8 * hlf + 2] += wj * a.z; acc[8 * hlf + 3] += wj * a.w;
-            acc[8 * hlf + 4] += wj * b.x; acc[8 * hlf + 5] += wj * b.y; acc[8 * hlf + 6] += wj * b.z; acc[8 * hlf + 7] += wj * b.w;
+      for (int u = 0; u < kMergeU; ++u) wj[u] = (j0 + u < n_parts) ? w[j0 + u] * inv : 0.f;
+      if (kF32) {
+        float4 v[kMergeU][4];
+        const float* src = reinterpret_cast<const float*>(O_part) + ((int64_t)j0 * n_rh + rh) * 512 + 8 * lane;
+#pragma unroll
+        for (int u = 0; u < kMergeU; ++u)
+          if (j0 + u < n_parts) {
+            v[u][0] = __ldcs(reinterpret_cast<const float4*>(src + u * part_stride));
+            v[u][1] = __ldcs(reinterpret_cast<const float4*>(src + u * part_stride + 4));
+            v[u][2] = __ldcs(reinterpret_cast<const float4*>(src + u * part_stride + 256));
+            v[u][3] = __ldcs(reinterpret_cast<const float4*>(src + u * part_stride + 260));
           }
-        } else {
-          const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(O_part) + ((int64_t)j * n_rh + rh) * 512;
 #pragma unroll
-          for (int hlf = 0; hlf < 2; ++hlf) {
-            const uint4 v = __ldcs(reinterpret_cast<const uint4*>(src + 256 * hlf + 8 * lane));
-            float f[8];
-            unpack8(v, f);
+        for (int u = 0; u < kMergeU; ++u)
+          if (wj[u] > 0.f) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[8 * hlf + e] += wj * f[e];
+            for (int q = 0; q < 4; ++q) {
+              acc[4 * q + 0] += wj[u] * v[u][q].x; acc[4 * q + 1] += wj[u] * v[u][q].y;
+              acc[4 * q + 2] += wj[u] * v[u][q].z; acc[4 * q + 3] += wj[u] * v[u][q].w;
+            }
           }
-        }
+      } else {
+        uint4 v[kMergeU][2];
+        const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(O_part) + ((int64_t)j0 * n_rh + rh) * 512 + 8 * lane;
+#pragma unroll
+        for (int u = 0; u < kMergeU; ++u)
+          if (j0 + u < n_parts) {
+            v[u][0] = __ldcs(reinterpret_cast<const uint4*>(src + u * part_stride));
+            v[u][1] = __ldcs(reinterpret_cast<const uint4*>(src + u * part_stride + 256));
+          }
+#pragma unroll
+        for (int u = 0; u < kMergeU; ++u)
+          if (wj[u] > 0.f) {
+            float f[16];
+            unpack8(v[u][0], f);
+            unpack8(v[u][1], f + 8);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) acc[e] += wj[u] * f[e];
+          }
       }
     }
     __nv_bfloat16* dst = O + rh * 512;
@@ -301,7 +339,7 @@ cudaError_t launch_relocate(const void* q_rope, int64_t n_rows, int32_t n_heads,
                             int sm_count, cudaStream_t stream) {
   const int64_t items = n_rows * n_heads * 8;
   if (items == 0 || seg_end <= seg_begin) return cudaSuccess;
-  rk_relocate_kernel<<<grid_for(items, sm_count, 8), 256, 0, stream>>>(
+  rk_relocate_kernel<<<grid_for((items + kRelU - 1) / kRelU, sm_count, 8), 256, 0, stream>>>(
       reinterpret_cast<const __nv_bfloat16*>(q_rope), n_rows, n_heads, row_stride, head_stride, seg_cs, seg_begin,
       seg_end - seg_begin, reinterpret_cast<__nv_bfloat16*>(out));
   return cudaGetLastError();
@@ -311,7 +349,8 @@ cudaError_t launch_merge(int32_t n_parts, int64_t n_rh, const void* O_part, int3
                          void* O, float* lse, int sm_count, cudaStream_t stream) {
   if (n_rh == 0) return cudaSuccess;
   const size_t smem = (size_t)8 * n_parts * sizeof(float);
-  const int grid = grid_for(n_rh * 32, sm_count, 8);
+  // persistent warps: as many blocks as stay resident with four parts' loads in registers (80 / 123 registers)
+  const int grid = grid_for(n_rh * 32, sm_count, part_dtype == 1 ? 2 : 3);
   if (part_dtype == 1)
     rk_merge_kernel<true><<<grid, 256, smem, stream>>>(n_parts, n_rh, O_part, lse_part,
                                                         reinterpret_cast<__nv_bfloat16*>(O), lse);

@@ -143,6 +143,12 @@ def test_moe_fanout_edge_cases(ctx):
     before = dev.clone()
     k, keep = ctx.rk_moe_fanout(dev, 0.0)                      # any three experts reach a zero threshold
     assert (k == 3).all() and torch.equal(dev, before)          # the weights are not touched
+    # weights that start 24 bytes into an allocation (8-byte aligned only) and a token count of 4n + 3
+    k_all, keep_all = ctx.rk_moe_fanout(dev, 0.8)
+    k_off, keep_off = ctx.rk_moe_fanout(dev[1:], 0.8)
+    assert torch.equal(k_off, k_all[1:]) and torch.equal(keep_off, keep_all[1:])
+    kw, keepw = policy.moe_fanout(p, 0.8)
+    assert np.array_equal(k_all.cpu().numpy(), kw) and np.array_equal(keep_all.cpu().numpy(), keepw)
     k0, keep0 = ctx.rk_moe_fanout(torch.empty((0, 6), dtype=torch.float32, device="cuda"), 0.8)
     assert k0.numel() == 0
     geo = torch.tensor([[4, 32, 1, 8, 16, 2]], dtype=torch.float32, device="cuda")
