@@ -34,12 +34,15 @@ from paper_2609_07008_b200 import dist as rkdist  # noqa: E402
 
 FLOP_PER_PAIR = 2 * 576 + 2 * 512     # QK^T over 576 + PV over 512 per visible (row, key, head)
 # dram__bytes_read.sum + dram__bytes_write.sum of the attention kernel's two launches per step, from the
-# one-pass ncu captures summarised under profiles/ (bytes per step; None where no capture exists)
+# one-pass ncu captures summarised under profiles/ (bytes per step; None where no capture exists).  bench.py
+# cannot run ncu itself: the figure is the capture's, taken on the kernel named in `captured_on`.
 PROFILED_DRAM_TRAFFIC = {
-    "flash256k": dict(bytes=37.44e9 + 9.58e9, algorithmic=4.91e9 + 1.20e9,
-                      source="profiles/attn_kernel_flash256k_dram_traffic.md"),
-    "flash1": dict(bytes=(352.0e6 + 224.9e6) + (169.6e6 + 74.8e6), algorithmic=(350.3e6 + 277.9e6) + (168.4e6 + 115.5e6),
-                   source="profiles/attn_kernel_flash1_ncu_full.md"),
+    "flash256k": dict(bytes=37.41e9 + 9.24e9, algorithmic=4.91e9 + 1.20e9,
+                      source="profiles/attn_kernel_flash256k_dram_traffic.md",
+                      captured_on="rk_mla_attn_kernel<kPhase=0, kStarve=0> (template instantiations, no run-time switches)"),
+    "flash1": dict(bytes=(352.5e6 + 224.8e6) + (169.3e6 + 74.4e6), algorithmic=(350.3e6 + 277.9e6) + (168.4e6 + 115.5e6),
+                   source="profiles/attn_kernel_flash1_ncu_full.md",
+                   captured_on="rk_mla_attn_kernel<kPhase=0, kStarve=0> (template instantiations, no run-time switches)"),
 }
 L2_BYTES = 126 * 1024 * 1024
 
@@ -114,6 +117,9 @@ class NvmlClock(threading.Thread):
         return v[len(v) // 2] if v else None
 
 
+AUX_SCALE = 1.0      # --aux-scale: shortens the steady-state loops (profiler runs)
+
+
 def timed_region(fn, stream, gpu_index, min_ms=300.0, lead_ms=30.0):
     """Times one call `fn` in its steady state: the same call is first repeated for at least lead_ms, then
     timed back to back (CUDA events on the launching stream) over at least 20 repeats and min_ms, with the
@@ -124,9 +130,9 @@ def timed_region(fn, stream, gpu_index, min_ms=300.0, lead_ms=30.0):
     b.record(stream)
     torch.cuda.synchronize()
     one = max(a.elapsed_time(b), 1e-3)
-    for _ in range(max(3, int(lead_ms / one))):
+    for _ in range(max(3, int(lead_ms * AUX_SCALE / one))):
         fn()
-    reps = max(20, int(min_ms / one))
+    reps = max(20 if AUX_SCALE >= 1.0 else 3, int(min_ms * AUX_SCALE / one))
     clk = NvmlClock(gpu_index)
     torch.cuda.synchronize()
     clk.start()
@@ -377,12 +383,17 @@ def main():
                          "the inverse output RoPE inside the attention kernel), W_uv 576 wide")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-aux", action="store_true", help="skip the standalone relocation / merge timings")
+    ap.add_argument("--aux-scale", type=float, default=1.0,
+                    help="scales the length of the steady-state timing loops of the standalone kernels and of the "
+                         "projection breakdown (1 = at least 20 repeats over 150-300 ms; a profiler run uses 0.01)")
     ap.add_argument("--with-offline", action="store_true", help="also time the offline artifact build")
     ap.add_argument("--layers", type=int, default=0,
                     help="independent layer invocations per step (own values and protected rows each; "
                          "default 37 for flash32k, the 3F-37R-3F stack, else 1)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rk" else args.warmup
+    global AUX_SCALE
+    AUX_SCALE = args.aux_scale
 
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # started plainly: bring up one rank per GPU ourselves (the same launch torch.distributed.run does)
@@ -526,10 +537,12 @@ def main():
                                                      bufs["y"]))
         width = prof.n_groups * prof.o_rank
         comb_bytes = 3 * req.T * width * 2
-        breakdown = dict(sliced_proj_ms=t_proj, sliced_proj_tflops=fl_proj / t_proj / 1e9,
+        _, fl_proj0, fl_wb0 = algorithmic_flops(prof, req, args.value_phase)      # layer 0 alone is timed here
+        breakdown = dict(sliced_proj_ms=t_proj, sliced_proj_tflops=fl_proj0 / t_proj / 1e9,
                          combine_ms=t_comb, combine_gbs=comb_bytes / t_comb / 1e6,
-                         wb_gemm_ms=t_cwb - t_comb, wb_gemm_tflops=fl_wb / (t_cwb - t_comb) / 1e9,
-                         wb_gemm_frac_of_nominal=fl_wb / (t_cwb - t_comb) / 1e9 / 2250.0)
+                         wb_gemm_ms=t_cwb - t_comb, wb_gemm_tflops=fl_wb0 / (t_cwb - t_comb) / 1e9,
+                         wb_gemm_frac_of_nominal=fl_wb0 / (t_cwb - t_comb) / 1e9 / 2250.0,
+                         note="each call repeated back to back for >= 150 ms (steady state under the power cap)")
         ctx.rk_poll_status()
 
     offline = None
@@ -551,6 +564,7 @@ def main():
                     ms_global_pass=float(np.mean(attn_g_ms)),
                     traffic=None if args.value_phase else (PROFILED_DRAM_TRAFFIC.get(name) or {}).get("bytes"),
                     traffic_note=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("source", "no ncu capture of this workload"),
+                    traffic_captured_on=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("captured_on"),
                     algorithmic_dram_bytes=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("algorithmic"))
     rest_tflops = (fl_proj + fl_wb) / (np.mean(rest_ms) * 1e-3) / 1e12
 

@@ -111,7 +111,8 @@ rk_status rk_create_ex(const rk_profile* profile, uint32_t flags, rk_ctx** out);
 rk_status rk_destroy(rk_ctx* ctx);
 /* Message of the last failing call on this context (valid until the next call). */
 const char* rk_last_error(const rk_ctx* ctx);
-/* Synchronises `stream`, returns the device status word (RK_OK or RK_ERR_TIMEOUT) and clears it. */
+/* Synchronises `stream`, returns the device status word (RK_OK, RK_ERR_TIMEOUT, or RK_ERR_ROWS from the
+ * bounds-checked build) and clears it. */
 rk_status rk_poll_status(rk_ctx* ctx, void* stream);
 /* Per-wait time limit of device-side waits, in milliseconds (default 2000). */
 rk_status rk_set_wait_limit_ms(rk_ctx* ctx, int32_t ms);
@@ -121,6 +122,14 @@ rk_status rk_set_wait_limit_ms(rk_ctx* ctx, int32_t ms);
  * rk_poll_status() reports RK_ERR_TIMEOUT.  Results are not produced while it is on.  Use it
  * together with a short rk_set_wait_limit_ms. */
 rk_status rk_test_starve_loads(rk_ctx* ctx, int32_t on);
+/* The library can be built with -DRK_CHECK (paper_2609_07008_b200/build.py, check=True): its kernels then
+ * test every index they derive from a request table (protected-row list, inverse row map, work list,
+ * compaction offsets) before using it, skip the access when it is out of range and record RK_ERR_ROWS in
+ * the status word that rk_poll_status reads.  It is a debugging aid for small cases, not the production
+ * build.  rk_check_selftest pushes one deliberately bad index through that check (nothing is accessed):
+ * on the checking build the next rk_poll_status returns RK_ERR_ROWS; the ordinary build returns
+ * RK_ERR_UNSUPPORTED here. */
+rk_status rk_check_selftest(rk_ctx* ctx, void* stream);
 
 /* Request geometry object: validates the layout and the protected-row list (Eq. protected;
  * the list is data here), builds row positions, per-segment relocation tables

@@ -54,7 +54,7 @@ class rk_layer_io(C.Structure):
 
 
 EXPORTS = ["rk_version", "rk_status_string", "rk_create", "rk_destroy", "rk_last_error", "rk_poll_status",
-           "rk_create_ex", "rk_segmented_merge_phase", "rk_set_wait_limit_ms", "rk_test_starve_loads", "rk_request_create", "rk_request_destroy", "rk_check_request",
+           "rk_create_ex", "rk_segmented_merge_phase", "rk_check_selftest", "rk_set_wait_limit_ms", "rk_test_starve_loads", "rk_request_create", "rk_request_destroy", "rk_check_request",
            "rk_request_get_info", "rk_workspace_bytes", "rk_relocate_q", "rk_mla_online_attn",
            "rk_segmented_merge", "rk_group_sliced_proj", "rk_group_sliced_proj_static", "rk_combine_offline",
            "rk_layer_host", "rk_layer_stack_host", "rk_mla_off_workspace_bytes", "rk_mla_off_build",
@@ -62,7 +62,8 @@ EXPORTS = ["rk_version", "rk_status_string", "rk_create", "rk_destroy", "rk_last
 
 
 def _load() -> C.CDLL:
-    path = _build.LIB_PATH
+    # RK_LIBRARY_PATH selects another build of the same library (the bounds-checked one, librk_check.so)
+    path = os.environ.get("RK_LIBRARY_PATH") or _build.LIB_PATH
     if not os.path.exists(path):
         raise RuntimeError(f"{path} is missing: build it with `python paper_2609_07008_b200/build.py` "
                            "(there is no fallback path)")
@@ -78,6 +79,7 @@ def _load() -> C.CDLL:
     lib.rk_poll_status.argtypes = [vp, vp]
     lib.rk_set_wait_limit_ms.argtypes = [vp, i32]
     lib.rk_test_starve_loads.argtypes = [vp, i32]
+    lib.rk_check_selftest.argtypes = [vp, vp]
     lib.rk_create_ex.argtypes = [C.POINTER(rk_profile), C.c_uint32, C.POINTER(vp)]
     lib.rk_segmented_merge_phase.argtypes = [vp, vp, i32, i32, i64, i32, vp, i32, vp, vp, vp, vp, vp]
     lib.rk_request_create.argtypes = [vp, C.POINTER(rk_layout), C.POINTER(i32), i64, C.POINTER(vp)]
@@ -195,6 +197,9 @@ class Context:
 
     def rk_set_wait_limit_ms(self, ms: int):
         self.check(lib.rk_set_wait_limit_ms(self.handle, ms))
+
+    def rk_check_selftest(self):
+        self.check(lib.rk_check_selftest(self.handle, _stream()))
 
     def rk_test_starve_loads(self, on: bool):
         self.check(lib.rk_test_starve_loads(self.handle, 1 if on else 0))

@@ -10,6 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "librk.so")
+CHECK_LIB_PATH = os.path.join(LIB_DIR, "librk_check.so")   # the same sources with -DRK_CHECK (device index checks)
 SOURCES = ["rk_host.cu", "rk_attn.cu", "rk_gemm.cu", "rk_stream.cu", "rk_policy.cu"]
 HEADERS = ["rk_ptx.cuh", "rk_internal.h", os.path.join("..", "..", "include", "rk.h")]
 
@@ -33,16 +34,22 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps if os.path.exists(d))
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
-        return LIB_PATH
+def build_library(force: bool = False, verbose: bool = False, check: bool = False) -> str:
+    """check=True builds librk_check.so: the same sources with -DRK_CHECK, whose kernels test every index they
+    derive from a request table and report a bad one through the status word (a debugging aid for small cases)."""
+    out_path = CHECK_LIB_PATH if check else LIB_PATH
+    if not force and not needs_build() and os.path.exists(out_path) and \
+            os.path.getmtime(out_path) >= os.path.getmtime(LIB_PATH):
+        return out_path
     os.makedirs(LIB_DIR, exist_ok=True)
     objs = []
     procs = []
     for src in _sources():
-        obj = os.path.join(LIB_DIR, src.replace(".cu", ".o"))
+        obj = os.path.join(LIB_DIR, src.replace(".cu", "_check.o" if check else ".o"))
         cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
                "-Xcompiler", "-fPIC", "-c", os.path.join(CSRC, src), "-o", obj]
+        if check:
+            cmd.append("-DRK_CHECK")
         if verbose:
             cmd += ["-Xptxas", "-v"]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
@@ -55,12 +62,12 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    link = [_nvcc(), "-shared", "-o", LIB_PATH] + objs
+    link = [_nvcc(), "-shared", "-o", out_path] + objs
     r = subprocess.run(link, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
     if r.returncode != 0:
         sys.stderr.write(r.stdout)
         raise RuntimeError("link failed")
-    return LIB_PATH
+    return out_path
 
 
 def ensure_built() -> str:
@@ -70,4 +77,4 @@ def ensure_built() -> str:
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv, check="--check" in sys.argv))

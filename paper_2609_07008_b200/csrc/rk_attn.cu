@@ -648,12 +648,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
     for (int w = pair; w < p.n_tiles && ok; w += p.n_pairs) {
       const AttnWorkItem item = get_work(p, w);
       const int r = item.tile * kAttnRowsPerPair + (int)crank * kAttnRowsPerCta + m;
-      const bool valid = r < p.n_flat;
+      bool valid = rk_index_ok(item.tile >= 0 && (long long)item.tile * kAttnRowsPerPair < p.n_flat, p.status,
+                               RK_CHK_WORK_TILE, item.tile) && r < p.n_flat;
       int pos = -1, prow = -1;
       if (valid) {
         const int tok = r / p.hpt;
         prow = p.rowmap ? p.rowmap[tok] : p.row_base + tok;
-        pos = p.row_pos[prow];
+        if (rk_index_ok(prow >= 0 && prow < p.n_rows_total, p.status, RK_CHK_PROT_ROW, prow))
+          pos = p.row_pos[prow];
+        else
+          valid = false;  // bounds-checked build: the row is skipped, nothing is read or written for it
       }
       float m_run = -INFINITY, l_run = 0.f;
       int kt = 0;

@@ -242,19 +242,244 @@ __global__ void __launch_bounds__(kGemmThreads, 1) rk_gemm_kernel(const __grid_c
   }
 }
 
+// ------------------------------------------------------------------------------------------------------
+// CTA-pair form for single-batch launches with N a multiple of 256 (the shared second projection W_b):
+// a cluster of two CTAs owns a 256 x 256 output tile, 128 rows each, and one cta_group::2 UMMA
+// (M = 256, N = 256, K = 16) per step reads A from both CTAs and one half of the B tile from each.  Every SM
+// then streams 16 KB of A and 16 KB of B per k-chunk instead of 16 + 32 KB: a third less L2 -> shared
+// memory traffic and shared-memory operand reads per flop at the same MMA rate, which under the board's
+// power limit is clock.  No multicast load is involved: each CTA fetches its own half of B with its own TMA.
+// ------------------------------------------------------------------------------------------------------
+constexpr int kPairStages = 5;
+struct PairSmem {
+  static constexpr uint32_t kABytes = kBM * kBK * 2;  // this CTA's 128 rows of A: 16 KB
+  static constexpr uint32_t kBBytes = 128 * kBK * 2;  // this CTA's 128 of the tile's 256 B rows: 16 KB
+  static constexpr uint32_t kStageBytes = kABytes + kBBytes;
+  static constexpr uint32_t kOffCStage = kPairStages * kStageBytes;
+  static constexpr uint32_t kCStageBytes = kBM * 128;
+  static constexpr uint32_t kOffBars = kOffCStage + 2 * kCStageBytes;
+  // full[kPairStages], empty[kPairStages], acc_full[2], acc_empty[2]
+  static constexpr uint32_t kOffTmemPtr = kOffBars + (2 * kPairStages + 4) * 8;
+  static constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
+  static constexpr uint32_t kBytes = kOffAbort + 8 + 1024;
+};
+
+// tile order: bands of kBandRows / 2 row-pair blocks, inside a band column tile first (see tile_coords)
+__device__ __forceinline__ void pair_tile_coords(int t, int n_pair_blocks, int n_tiles_n, int& pb, int& nt) {
+  constexpr int kBand = kBandRows / 2;
+  const int per_band = kBand * n_tiles_n;
+  const int band = t / per_band;
+  const int rows_here = min(kBand, n_pair_blocks - band * kBand);
+  const int rem = t - band * per_band;
+  nt = rem / rows_here;
+  pb = band * kBand + (rem - nt * rows_here);
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+    rk_gemm_pair_kernel(const __grid_constant__ GemmParams p) {
+  using S = PairSmem;
+  constexpr int BN = 256;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t crank = cluster_ctarank();
+  const bool leader = (crank == 0);
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  auto full_bar = [&](int s) -> uint32_t { return smem_base + S::kOffBars + 8u * s; };
+  auto empty_bar = [&](int s) -> uint32_t { return smem_base + S::kOffBars + 8u * (kPairStages + s); };
+  auto acc_full_bar = [&](int b) -> uint32_t { return smem_base + S::kOffBars + 8u * (2 * kPairStages + b); };
+  auto acc_empty_bar = [&](int b) -> uint32_t { return smem_base + S::kOffBars + 8u * (2 * kPairStages + 2 + b); };
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::kOffAbort);
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + S::kOffTmemPtr);
+  const uint64_t limit = p.wait_ns;
+
+  const int n_tiles_n = p.N / BN;
+  const int n_pair_blocks = (p.M + 2 * kBM - 1) / (2 * kBM);
+  const int n_tiles = n_tiles_n * n_pair_blocks;
+  const int k_chunks = p.K / kBK;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < kPairStages; ++s) {
+      mbar_init(full_bar(s), 1);   // leader's: one arrival (its own expect_tx) + the bytes of both CTAs
+      mbar_init(empty_bar(s), 1);  // each CTA's: the pair's commit arrives on both
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(acc_full_bar(b), 1);   // each CTA's: the pair's commit arrives on both
+      mbar_init(acc_empty_bar(b), 8);  // leader's: the four epilogue warps of both CTAs
+    }
+    fence_mbar_init_cluster();
+  }
+  if (warp == 0) {
+    __syncwarp();
+    tmem_alloc<2>(smem_base + S::kOffTmemPtr, 512);
+    tmem_relinquish<2>();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_ptr_smem;
+
+  if (warp == 0) {
+    // ---- TMA producer: this CTA's A rows and its half of the B tile; bytes are counted on the leader's barrier ----
+    if (lane == 0) {
+      tma_prefetch_desc(&p.tm_a);
+      tma_prefetch_desc(&p.tm_b);
+    }
+    const GemmBatch bt = p.batches[0];
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = pair; t < n_tiles && ok; t += n_pairs) {
+      int pb, nt;
+      pair_tile_coords(t, n_pair_blocks, n_tiles_n, pb, nt);
+      const int m0 = pb * 2 * kBM + (int)crank * kBM, n0 = nt * BN + (int)crank * 128;
+      for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
+        const uint32_t s = it % kPairStages;
+        if (it >= (uint32_t)kPairStages)
+          ok = mbar_wait_bounded<false>(empty_bar(s), ((it / kPairStages) & 1u) ^ 1u, limit, abort_flag, p.status, WG_EMPTY, t);
+        if (!ok) break;
+        if (elect_one()) {
+          if (leader) mbar_arrive_expect_tx(full_bar(s), 2 * S::kStageBytes);
+          const uint32_t full_remote = mapa_shared(full_bar(s), 0);
+          const int k = kc * kBK;
+          const uint32_t a_dst = smem_base + s * S::kStageBytes;
+          tma_load_2d_pair(a_dst, &p.tm_a, full_remote, bt.a_col0 + k, m0);
+          tma_load_2d_pair(a_dst + S::kABytes, &p.tm_b, full_remote, bt.b_col0 + k, bt.b_row0 + n0);
+        }
+        __syncwarp();
+      }
+    }
+    for (uint32_t back = 1; back <= (uint32_t)kPairStages && ok; ++back) {
+      if (it >= back) {
+        const uint32_t u = it - back;
+        ok = mbar_wait_bounded<false>(empty_bar(u % kPairStages), (u / kPairStages) & 1u, limit, abort_flag, p.status, WG_EMPTY, -1);
+      }
+    }
+  } else if (warp == 1) {
+    // ---- UMMA issuer (leader CTA only) ----
+    if (leader) {
+      constexpr uint32_t idesc = umma_idesc_bf16(2 * kBM, BN, 0, 0);
+      uint32_t it = 0, tile_i = 0;
+      bool ok = true;
+      for (int t = pair; t < n_tiles && ok; t += n_pairs, ++tile_i) {
+        const uint32_t b = tile_i & 1u;
+        if (tile_i >= 2) {
+          ok = mbar_wait_bounded<true>(acc_empty_bar(b), ((tile_i >> 1) & 1u) ^ 1u, limit, abort_flag, p.status, WG_ACC_EMPTY, t);
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
+        const uint32_t tmem_acc = tmem_base + b * BN;
+        for (int kc = 0; kc < k_chunks && ok; ++kc, ++it) {
+          const uint32_t s = it % kPairStages;
+          ok = mbar_wait_bounded<false>(full_bar(s), (it / kPairStages) & 1u, limit, abort_flag, p.status, WG_FULL, t);
+          if (!ok) break;
+          const uint32_t a_addr = smem_base + s * S::kStageBytes;
+          const uint32_t b_addr = a_addr + S::kABytes;
+          if (elect_one()) {
+            const uint64_t da = umma_desc_sw128(a_addr, 16, 1024), db = umma_desc_sw128(b_addr, 16, 1024);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma_f16<2>(tmem_acc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kc > 0 || k > 0) ? 1u : 0u);
+            umma_commit_2_mc(empty_bar(s), 3);
+            if (kc == k_chunks - 1) umma_commit_2_mc(acc_full_bar(b), 3);
+          }
+          __syncwarp();
+        }
+      }
+    }
+  } else if (warp >= 4) {
+    // ---- epilogue: this CTA's 128 rows of the accumulator (lane = row, 256 columns) ----
+    const int L = threadIdx.x - 128;
+    const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
+    const uint32_t acc_empty_remote = mapa_shared(acc_empty_bar(0), 0);
+    uint32_t tile_i = 0, chunk_i = 0;
+    bool ok = true;
+    if (L == 0) tma_prefetch_desc(&p.tm_c);
+    const GemmBatch bt = p.batches[0];
+    for (int t = pair; t < n_tiles && ok; t += n_pairs, ++tile_i) {
+      const uint32_t b = tile_i & 1u;
+      int pb, nt;
+      pair_tile_coords(t, n_pair_blocks, n_tiles_n, pb, nt);
+      const int m0 = pb * 2 * kBM + (int)crank * kBM, n0 = nt * BN;
+      ok = mbar_wait_bounded<false>(acc_full_bar(b), (tile_i >> 1) & 1u, limit, abort_flag, p.status, WG_ACC_FULL, t);
+      ok = named_barrier_and(1, 128, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+#pragma unroll 1
+      for (int cc = 0; cc < BN; cc += 64, ++chunk_i) {
+        uint32_t o[64];
+        tmem_ld_x32(tmem_base + lane_base + b * BN + cc, o);
+        tmem_ld_x32(tmem_base + lane_base + b * BN + cc + 32, o + 32);
+        tmem_wait_ld();
+        if (cc + 64 >= BN) {  // the accumulator is in registers: hand it back to the tensor cores of the pair
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_remote(acc_empty_remote + 8u * b);
+        }
+        const uint32_t buf = chunk_i & 1u;
+        if (L == 0) bulk_wait_group_read<1>();
+        named_barrier_sync(1, 128);
+        uint8_t* stage = smem + S::kOffCStage + buf * S::kCStageBytes;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(o[8 * e + 0]), __uint_as_float(o[8 * e + 1]));
+          v.y = pack_bf16(__uint_as_float(o[8 * e + 2]), __uint_as_float(o[8 * e + 3]));
+          v.z = pack_bf16(__uint_as_float(o[8 * e + 4]), __uint_as_float(o[8 * e + 5]));
+          v.w = pack_bf16(__uint_as_float(o[8 * e + 6]), __uint_as_float(o[8 * e + 7]));
+          *reinterpret_cast<uint4*>(stage + sw128_offset((uint32_t)L, (uint32_t)e)) = v;
+        }
+        fence_proxy_async_smem();
+        named_barrier_sync(1, 128);
+        if (L == 0 && m0 < p.M) {
+          tma_store_2d(&p.tm_c, smem_base + S::kOffCStage + buf * S::kCStageBytes, bt.c_col0 + n0 + cc, m0);
+          bulk_commit_group();
+        }
+      }
+    }
+    if (L == 0) bulk_wait_group<0>();
+  }
+  if (*abort_flag != 0) {
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+  }
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  if (warp == 0) {
+    __syncwarp();
+    tmem_dealloc<2>(tmem_base, 512);
+  }
+}
+
 }  // namespace
+
+bool gemm_uses_pairs(int M, int N, int n_batches) { return n_batches == 1 && N % 256 == 0 && M >= 512; }
 
 cudaError_t gemm_setup() {
   cudaError_t e = cudaFuncSetAttribute(rk_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)GemmSmem<128>::kBytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(rk_gemm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)GemmSmem<256>::kBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(rk_gemm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GemmSmem<256>::kBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(rk_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PairSmem::kBytes);
+  return e;
 }
 
 cudaError_t launch_gemm(const GemmParams& p, int bn, int sm_count, cudaStream_t stream) {
   const long long tiles = (long long)((p.N + bn - 1) / bn) * ((p.M + kBM - 1) / kBM) * p.n_batches;
   if (tiles <= 0) return cudaSuccess;
+  if (gemm_uses_pairs(p.M, p.N, p.n_batches)) {  // CTA pairs over 256 x 256 tiles (tm_b's box is 128 rows then)
+    const long long pair_tiles = (long long)(p.N / 256) * ((p.M + 2 * kBM - 1) / (2 * kBM));
+    const int n_pairs = (int)(pair_tiles < sm_count / 2 ? pair_tiles : sm_count / 2);
+    rk_gemm_pair_kernel<<<2 * n_pairs, kGemmThreads, PairSmem::kBytes, stream>>>(p);
+    return cudaGetLastError();
+  }
   const int grid = (int)(tiles < sm_count ? tiles : sm_count);
   if (bn == 128)
     rk_gemm_kernel<128><<<grid, kGemmThreads, GemmSmem<128>::kBytes, stream>>>(p);

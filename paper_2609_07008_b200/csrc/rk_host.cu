@@ -351,6 +351,16 @@ rk_status rk_set_wait_limit_ms(rk_ctx* ctx, int32_t ms) {
   return RK_OK;
 }
 
+rk_status rk_check_selftest(rk_ctx* ctx, void* stream) {
+  if (!ctx) return RK_ERR_NULL;
+  cudaError_t e = launch_check_selftest(ctx->d_status, reinterpret_cast<cudaStream_t>(stream));
+  if (e == cudaErrorNotSupported) {
+    cudaGetLastError();
+    return fail(ctx, RK_ERR_UNSUPPORTED, "this library was built without the device index checks (-DRK_CHECK)");
+  }
+  return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "self-test launch");
+}
+
 rk_status rk_test_starve_loads(rk_ctx* ctx, int32_t on) {
   if (!ctx) return RK_ERR_NULL;
   ctx->starve_loads = on != 0;
@@ -366,6 +376,8 @@ rk_status rk_poll_status(rk_ctx* ctx, void* stream) {
   if (e != cudaSuccess) return cuda_fail(ctx, e, "status readback");
   if (h.code != 0) {
     cudaMemset(ctx->d_status, 0, sizeof(DeviceStatus));
+    if (h.code == RK_ERR_ROWS)  // only the bounds-checked build reports this
+      return fail(ctx, RK_ERR_ROWS, "device index check failed: table %d, block %d, value %d", h.where, h.block, h.aux);
     return fail(ctx, RK_ERR_TIMEOUT, "device wait expired: tag %d, block %d, aux %d", h.where, h.block, h.aux);
   }
   return RK_OK;
@@ -639,6 +651,7 @@ static rk_status attn_pass(rk_ctx* ctx, const rk_request* rq, const void* kv, co
   p.scale_log2 = ctx->prof.sm_scale * 1.44269504088896340736f;
   p.isolated = isolated;
   p.row_base = (int32_t)row_base;
+  p.n_rows_total = (int32_t)rq->T;
   memcpy(p.rope_turns, ctx->rope_turns, sizeof(p.rope_turns));
   cudaError_t e = launch_attention(p, n_pairs, ctx->value_phase, ctx->starve_loads, stream);
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "attention launch");
@@ -748,7 +761,8 @@ static rk_status run_gemm(rk_ctx* ctx, const void* A, int64_t a_rows, int64_t a_
   const int bn = (N % 256 == 0) ? 256 : 128;
   rk_status s = make_tmap(ctx, &p.tm_a, A, (uint64_t)a_rows, (uint64_t)a_cols, (uint64_t)a_cols, 64, 128);
   if (s != RK_OK) return s;
-  s = make_tmap(ctx, &p.tm_b, B, (uint64_t)b_rows, (uint64_t)b_cols, (uint64_t)b_cols, 64, (uint32_t)bn);
+  s = make_tmap(ctx, &p.tm_b, B, (uint64_t)b_rows, (uint64_t)b_cols, (uint64_t)b_cols, 64,
+                gemm_uses_pairs(M, N, n_batches) ? 128u : (uint32_t)bn);
   if (s != RK_OK) return s;
   s = make_tmap(ctx, &p.tm_c, C, (uint64_t)M, (uint64_t)ldc, (uint64_t)ldc, 64, 128);
   if (s != RK_OK) return s;
@@ -814,7 +828,7 @@ rk_status rk_combine_offline(rk_ctx* ctx, const rk_request* rq, const void* z_on
     return fail(ctx, RK_ERR_ALIGN, "tensor base pointers must be 16-byte aligned");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const int64_t width = (int64_t)ctx->prof.n_groups * ctx->prof.o_rank;
-  cudaError_t e = launch_combine(z_on_g, z_on_l, z_off, rq->d_inv_map, rq->T, width, z, ctx->sm_count, st);
+  cudaError_t e = launch_combine(z_on_g, z_on_l, z_off, rq->d_inv_map, rq->T, width, z, rq->A, ctx->d_status, ctx->sm_count, st);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "combine launch");
   if (!W_b) return RK_OK;
   return run_gemm(ctx, z, rq->T, width, W_b, ctx->prof.d_model, width, y, ctx->prof.d_model, (int)rq->T,
@@ -887,7 +901,7 @@ static rk_status layer_compute(rk_ctx* ctx, const rk_request* rq, const rk_layer
       if (e != cudaSuccess) return cuda_fail(ctx, e, "stream wait");
     }
     e = launch_combine(zg + (size_t)r0 * width * 2, dev->z_on_l, zo ? zo + (size_t)r0 * width * 2 : nullptr, rq->d_inv_map + r0, n,
-                       (int64_t)width, zz + (size_t)r0 * width * 2, ctx->sm_count, st);
+                       (int64_t)width, zz + (size_t)r0 * width * 2, rq->A, ctx->d_status, ctx->sm_count, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "combine launch");
     s = run_gemm(ctx, zz + (size_t)r0 * width * 2, n, (int64_t)width, W_b, dm, (int64_t)width, yy + (size_t)r0 * dm * 2, dm, (int)n,
                  (int)dm, (int)width, ctx->off_wb, 1, st);
@@ -1078,6 +1092,7 @@ rk_status rk_protected_rows(rk_ctx* ctx, const rk_layout* lay, const rk_policy* 
   h.rows_out = rows_out;
   h.count_out = reinterpret_cast<long long*>(count_out);
   h.workspace = workspace;
+  h.status = ctx->d_status;
   cudaError_t e = launch_protected_rows(h, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(ctx, e, "protected-row kernels");
   return RK_OK;

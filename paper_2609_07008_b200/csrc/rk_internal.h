@@ -45,6 +45,7 @@ struct AttnParams {
   float scale_log2;  // sm_scale * log2(e)
   int32_t isolated;  // 1: a row sees only its own segment (documents built alone, Algorithm 1)
   int32_t row_base;  // packed row of token slot 0 when rowmap is null
+  int32_t n_rows_total;  // T: bound of every packed-row index (read by the bounds-checked build)
   double rope_turns[32];  // theta_j / (2 pi), j = 0..31 (used by the output-phase instantiation only)
 };
 
@@ -64,7 +65,7 @@ struct GemmBatch {
 
 struct GemmParams {
   CUtensorMap tm_a;  // [M rows][a_cols] box 64 x 128
-  CUtensorMap tm_b;  // [b_rows][b_cols] box 64 x BN
+  CUtensorMap tm_b;  // [b_rows][b_cols] box 64 x BN (64 x 128 for the CTA-pair kernel)
   CUtensorMap tm_c;  // [M rows][ldc] box 64 x 128 (epilogue stores)
   void* C;
   const GemmBatch* batches;
@@ -77,6 +78,8 @@ struct GemmParams {
 
 cudaError_t launch_gemm(const GemmParams& p, int bn, int sm_count, cudaStream_t stream);
 cudaError_t gemm_setup();
+// single-batch launches with N a multiple of 256 run on CTA pairs; their B tensor map needs a 128-row box
+bool gemm_uses_pairs(int M, int N, int n_batches);
 
 // ---- streaming kernels -----------------------------------------------------------------------
 constexpr int kMergeMaxParts = 4096;  // the merge keeps 8 warps x n_parts weights in shared memory (128 KB at most)
@@ -89,8 +92,9 @@ cudaError_t launch_merge(int32_t n_parts, int64_t n_rh, const void* O_part, int3
 cudaError_t launch_merge_phase(int32_t n_parts, int64_t n_rows, int32_t n_heads, const void* O_part, int32_t part_dtype,
                                const float* lse_part, const float2* seg_cs, const int32_t* row_pos, const double* rope_turns,
                                void* O, float* lse, int sm_count, cudaStream_t stream);
-cudaError_t launch_combine(const void* z_on_g, const void* z_on_l, const void* z_off, const int32_t* inv_map,
-                           int64_t T, int64_t width, void* z, int sm_count, cudaStream_t stream);
+cudaError_t launch_combine(const void* z_on_g, const void* z_on_l, const void* z_off, const int32_t* inv_map, int64_t T,
+                           int64_t width, void* z, int64_t n_prot, DeviceStatus* status, int sm_count, cudaStream_t stream);
+cudaError_t launch_check_selftest(DeviceStatus* status, cudaStream_t stream);  // does something in the bounds-checked build only
 
 // ---- selection rules (Eq. protected, Eq. moe) --------------------------------------------------
 constexpr uint8_t kPolicyStructural = 1, kPolicyCandidate = 2, kPolicyDirty = 4;
@@ -111,6 +115,7 @@ struct PolicyParams {
   unsigned* block_counts;
   int32_t* rows_out;
   long long* count_out;
+  DeviceStatus* status;
   long long req_end, tail_rows;
   int32_t n_segs, T, edge_rows, budget_bp;
 };
@@ -127,6 +132,7 @@ struct PolicyHost {
   int32_t* rows_out;
   long long* count_out;
   void* workspace;
+  DeviceStatus* status;
 };
 
 size_t policy_workspace_bytes(int64_t T, int32_t n_segs);

@@ -201,7 +201,10 @@ __global__ void __launch_bounds__(kPolicyThreads) policy_scatter_kernel(PolicyPa
     warp_sums[lane] = x - v;
   }
   __syncthreads();
-  if (sel) p.rows_out[p.block_counts[blockIdx.x] + warp_sums[warp] + __popc(ballot & ((1u << lane) - 1u))] = t;
+  if (sel) {
+    const unsigned at = p.block_counts[blockIdx.x] + warp_sums[warp] + __popc(ballot & ((1u << lane) - 1u));
+    if (rk_index_ok(at < (unsigned)p.T, p.status, RK_CHK_COMPACT, at)) p.rows_out[at] = t;
+  }
 }
 
 // Eq. (moe) for one token.  The six weights are sorted by a 12-exchange min/max network (values only:
@@ -323,6 +326,7 @@ cudaError_t launch_protected_rows(const PolicyHost& h, cudaStream_t stream) {
   p.scores = h.scores;
   p.rows_out = h.rows_out;
   p.count_out = h.count_out;
+  p.status = h.status;
 
   cudaError_t e;
   // h.seg_tab_host: [seg_off (S+1) | seg_delta (S)] as int32, h.has_host: [S]; both stay alive in the

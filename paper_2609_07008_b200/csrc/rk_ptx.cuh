@@ -29,6 +29,26 @@ __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where, int 
   }
 }
 
+// Bounds-checked build (-DRK_CHECK, a debugging aid: run the small cases on it): every index that device
+// code derives from a request table (protected-row list, inverse row map, work list, compaction offsets) is
+// tested before it is used; a bad one is recorded in the status word (code RK_ERR_ROWS, `where` names the
+// table, `aux` holds the value) and the access is skipped.  Nothing traps.  In the ordinary build the
+// function is the constant true and the test disappears.
+enum { RK_CHK_PROT_ROW = 101, RK_CHK_WORK_TILE = 102, RK_CHK_INV_MAP = 103, RK_CHK_COMPACT = 104, RK_CHK_SELFTEST = 199 };
+#ifdef RK_CHECK
+__device__ __forceinline__ bool rk_index_ok(bool ok, DeviceStatus* st, int where, long long value) {
+  if (!ok && st != nullptr && atomicCAS(&st->code, 0, 4 /*RK_ERR_ROWS*/) == 0) {
+    st->where = where;
+    st->block = (int)blockIdx.x;
+    st->aux = (int)value;
+    __threadfence();
+  }
+  return ok;
+}
+#else
+__device__ __forceinline__ bool rk_index_ok(bool, DeviceStatus*, int, long long) { return true; }
+#endif
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
