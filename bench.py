@@ -445,6 +445,7 @@ def main():
         if ev: ev[2].record(stream)
         ctx.rk_group_sliced_proj(r, bufs["O_g"], bufs["O_l"], wl.w_uv, wl.w_a, bufs["z_on_g"], bufs["z_on_l"],
                                  bufs["workspace"])
+        if ev: ev[4].record(stream)
         ctx.rk_combine_offline(r, bufs["z_on_g"], bufs["z_on_l"], wl.z_off, wl.w_b, bufs["z"], bufs["y"])
         if ev: ev[3].record(stream)
 
@@ -462,7 +463,7 @@ def main():
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    evs = [[[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_layers)]
+    evs = [[[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(n_layers)]
            for _ in range(args.steps)]
     rkdist.barrier()
     torch.cuda.synchronize()
@@ -477,6 +478,8 @@ def main():
     attn_ms = [sum(e[0].elapsed_time(e[2]) for e in evs[i]) for i in range(args.steps)]
     attn_g_ms = [sum(e[0].elapsed_time(e[1]) for e in evs[i]) for i in range(args.steps)]
     rest_ms = [sum(e[2].elapsed_time(e[3]) for e in evs[i]) for i in range(args.steps)]
+    proj_in_step_ms = float(np.mean([sum(e[2].elapsed_time(e[4]) for e in evs[i]) for i in range(args.steps)]))
+    comb_wb_in_step_ms = float(np.mean([sum(e[4].elapsed_time(e[3]) for e in evs[i]) for i in range(args.steps)]))
     total_ms = float(sum(step_ms))
     total_ms_max = rkdist.max_over_ranks(total_ms, dev)
     sampler.join(timeout=2)
@@ -542,7 +545,12 @@ def main():
                          combine_ms=t_comb, combine_gbs=comb_bytes / t_comb / 1e6,
                          wb_gemm_ms=t_cwb - t_comb, wb_gemm_tflops=fl_wb0 / (t_cwb - t_comb) / 1e9,
                          wb_gemm_frac_of_nominal=fl_wb0 / (t_cwb - t_comb) / 1e9 / 2250.0,
-                         note="each call repeated back to back for >= 150 ms (steady state under the power cap)")
+                         note="each call repeated back to back for >= 150 ms (steady state under the power cap)",
+                         # the same stages inside the timed steps (events between the calls; W_b = the combine + W_b call
+                         # minus the stand-alone combine time), at the clock the step itself runs at
+                         in_step_sliced_proj_ms=proj_in_step_ms / n_layers,
+                         in_step_combine_and_wb_ms=comb_wb_in_step_ms / n_layers,
+                         in_step_wb_gemm_tflops=fl_wb0 / max(comb_wb_in_step_ms / n_layers - t_comb, 1e-6) / 1e9)
         ctx.rk_poll_status()
 
     offline = None

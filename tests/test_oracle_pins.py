@@ -252,22 +252,27 @@ def test_p6_zero_query_running_mean_and_count():
 
 
 def test_p7_one_hot_limit():
+    """q = lambda K_req[k*] with k* the visible key of largest norm: its own score lambda |K*|^2 exceeds every other
+    score lambda <K*, K_k> (Cauchy-Schwarz, strict for non-parallel keys), so for large lambda the softmax puts all
+    weight on k* and the output is its latent c_{k*}; lse tends to the top score."""
     p = small_problem(14)
     pos = oracle.request_positions(p["seg_off"], p["seg_delta"])
     k_req = oracle.keys_in_request_frame(p["kv"], p["seg_off"], p["seg_delta"], p["d_c"], p["base"])
     v = p["kv"][:, :p["d_c"]]
     t = int(np.argmax(pos))                                          # sees everything
-    kstar = 4
-    # make k* the unique maximiser: q along K_req[k*] after removing what it shares with others
-    q = np.zeros((1, 1, p["d_c"] + p["d_r"]))
-    q[0, 0] = k_req[kstar] * 4000.0 / p["sm_scale"]
-    s = (k_req @ q[0, 0]) * p["sm_scale"]
-    if np.argmax(s) == kstar:
-        O, _ = oracle.attend_rows(q, pos[[t]], k_req, v, pos, p["sm_scale"])
-        assert np.allclose(O[0, 0], v[np.argmax(s)], atol=1e-6)
-    else:  # norm of another key dominates: the limit picks that key instead
-        O, _ = oracle.attend_rows(q, pos[[t]], k_req, v, pos, p["sm_scale"])
-        assert np.allclose(O[0, 0], v[np.argmax(s)], atol=1e-6)
+    kstar = int(np.argmax(np.linalg.norm(k_req, axis=1)))
+    lam = 4000.0 / p["sm_scale"]
+    q = (k_req[kstar] * lam)[None, None, :]
+    s_all = (k_req @ q[0, 0]) * p["sm_scale"]
+    assert int(np.argmax(s_all)) == kstar and np.sort(s_all)[-1] - np.sort(s_all)[-2] > 50.0
+    O, lse = oracle.attend_rows(q, pos[[t]], k_req, v, pos, p["sm_scale"])
+    assert np.allclose(O[0, 0], v[kstar], atol=1e-12)
+    assert abs(lse[0, 0] - s_all[kstar]) < 1e-9 * abs(s_all[kstar])
+    # a row that cannot see k* does not get its latent
+    hidden = np.nonzero(pos < pos[kstar])[0]
+    if len(hidden):
+        O2, _ = oracle.attend_rows(q, pos[hidden[:1]], k_req, v, pos, p["sm_scale"])
+        assert not np.allclose(O2[0, 0], v[kstar], atol=1e-3)
 
 
 # -- P8 / P9: invariances -----------------------------------------------------------------------
