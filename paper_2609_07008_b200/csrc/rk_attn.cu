@@ -38,20 +38,25 @@ constexpr uint32_t kStageBytes = 2 * kChunkBytes;
 constexpr uint32_t kQChunkBytes = 8192;  // 64 rows x 64 dims bf16
 
 // Two instantiations share this file.  The plain one (values = the 512-wide latent) keeps latent dims
-// 256-511 of the Q tile in tensor memory and runs a four-stage ring.  The output-phase one (values = the
-// whole stored row, latent and rope dims; Eq. offonline's inverse output RoPE, Algorithm 2's RestorePhase)
-// needs 32 more accumulator columns for the rope part of O, which do not fit beside the tensor-memory Q
-// half (256 + 128 + 128 + 32 > 512): it keeps all of Q in shared memory and runs a three-stage ring.
+// 256-511 of the Q tile in tensor memory (128 columns); that pays for the fourth stage of the ring.  The
+// output-phase one (values = the whole stored row, latent and rope dims; Eq. offonline's inverse output
+// RoPE, Algorithm 2's RestorePhase) needs 32 more accumulator columns for the rope part of O, so only 96
+// columns are left for Q: latent dims 320-511.  The 8 KB that its fifth shared-memory Q chunk costs come from
+// the pristine rope chunk, which in this instantiation lives in the relocation warp's registers (it lands in
+// the second rotated-rope buffer and is picked up from there at the start of a row tile).  Both run four stages.
 template <bool kPhase>
 struct Cfg {
-  static constexpr int kStages = kPhase ? 3 : 4;          // ring of 32 KB stages (two 16 KB TMA boxes each)
-  static constexpr int kQSmemChunks = kPhase ? 8 : 4;     // 64-dim latent chunks of Q kept in shared memory
+  static constexpr int kStages = 4;                       // ring of 32 KB stages (two 16 KB TMA boxes each)
+  static constexpr int kQSmemChunks = kPhase ? 5 : 4;     // 64-dim latent chunks of Q kept in shared memory
+  static constexpr int kQTmemChunks = 8 - kQSmemChunks;   // ... kept in tensor memory (32 columns each)
   static constexpr int kStagesPerKeyTile = kPhase ? 10 : 9;  // K: 5, V: 4, rope part of V: 1
   static constexpr int kOW = kPhase ? kDQK : kDLatent;    // width of an output row
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr uint32_t kOffQLat = 0;
-  static constexpr uint32_t kOffQPristine = kOffQLat + kQSmemChunks * kQChunkBytes;  // rope chunk as loaded
-  static constexpr uint32_t kOffQRot = kOffQPristine + kQChunkBytes;                 // 2 rotated rope chunks
+  // plain: rope chunk as loaded, then 2 rotated rope chunks.  output-phase: no buffer for the chunk as loaded;
+  // it lands in the second rotated buffer
+  static constexpr uint32_t kOffQRot = kOffQLat + (kQSmemChunks + (kPhase ? 0 : 1)) * kQChunkBytes;
+  static constexpr uint32_t kOffQPristine = kPhase ? kOffQRot + kQChunkBytes : kOffQLat + kQSmemChunks * kQChunkBytes;
   static constexpr uint32_t kOffP = kOffQRot + 2 * kQChunkBytes;                     // 4 sub-chunks [64 x 64 keys]
   static constexpr uint32_t kOffRing = kOffP + 4 * kQChunkBytes;
   static constexpr uint32_t kOffBars = kOffRing + kStages * kStageBytes;
@@ -72,6 +77,7 @@ constexpr uint32_t kColO = 0;     // two halves of 128 columns
 constexpr uint32_t kColS = 256;   // one 128-column score buffer
 constexpr uint32_t kColQ = 384;   // plain: latent dims 256-511 of the Q tile as a TMEM A operand (both lane halves hold the rows)
 constexpr uint32_t kColOr = 384;  // output-phase: the 64 rope dims of O (N = 64 folds onto 32 columns)
+constexpr uint32_t kColQp = 416;  // output-phase: latent dims 320-511 of the Q tile (96 columns)
 
 constexpr uint32_t kIdescQK = umma_idesc_bf16(128, 256, 0, 0);
 constexpr uint32_t kIdescPV = umma_idesc_bf16(128, 256, 0, 1);
@@ -362,10 +368,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         tma_load_2d_hint(smem_base + C::kOffQPristine, &p.tm_q, bar(C::kBarQFull), kDLatent, qrow, pol_q);
       }
       __syncwarp();
-      // Upper latent half (dims 256-511): staged through one ring stage, from where the softmax warps move
-      // it into tensor memory.  Each CTA loads its own rows and signals its own barrier; the issuer lets go
-      // of the ring position once both CTAs have finished the move.
-      if constexpr (!kPhase) {
+      // Upper latent part (dims 256-511, or 320-511): staged through one ring stage, from where the softmax
+      // warps move it into tensor memory.  Each CTA loads its own rows and signals its own barrier; the issuer
+      // lets go of the ring position once both CTAs have finished the move.
+      {
         const uint32_t s = rp.stage();
         if (rp.it >= (uint32_t)kStages) {
           ok = mbar_wait_bounded<false>(bar(C::kBarRingEmpty + s), rp.parity() ^ 1u, limit, abort_flag, p.status,
@@ -374,10 +380,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         }
         if (!kStarve && elect_one()) {
           if (leader) mbar_arrive(bar(C::kBarRingFull + s));  // keeps the ring's phases in step; no bytes land here
-          mbar_arrive_expect_tx(bar(C::kBarQhFull), 4 * kQChunkBytes);
-          for (int d = 0; d < 4; ++d)
+          mbar_arrive_expect_tx(bar(C::kBarQhFull), C::kQTmemChunks * kQChunkBytes);
+          for (int d = 0; d < C::kQTmemChunks; ++d)
             tma_load_2d_hint(smem_base + C::kOffRing + s * kStageBytes + d * kQChunkBytes, &p.tm_q, bar(C::kBarQhFull),
-                             256 + d * 64, qrow, pol_q);
+                             (C::kQSmemChunks + d) * 64, qrow, pol_q);
         }
         __syncwarp();
         rp.advance();
@@ -425,7 +431,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         const int n_kt = count_key_tiles(p, item);
         int kt_issued = 0;  // key tiles whose QK^T has been issued
         int kt_pv = 0;      // key tiles whose PV has been issued
-        if constexpr (!kPhase) {  // ring position of the staged upper Q half: wait for both CTAs' move into TMEM, then let go of it
+        {  // ring position of the staged upper Q part: wait for both CTAs' move into TMEM, then let go of it
           const uint32_t s = rp.stage();
           ok = mbar_wait_bounded<false>(bar(C::kBarRingFull + s), rp.parity(), limit, abort_flag, p.status, W_RINGFULL, w) &&
                mbar_wait_bounded<true>(bar(C::kBarQhDone), qh_done_phase, limit, abort_flag, p.status, W_QHDONE, w);
@@ -460,7 +466,22 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             }
             const uint32_t b_addr = smem_base + C::kOffRing + s * kStageBytes;
             if (elect_one()) {
-              if (!kPhase && st >= 2 && st < 4) {  // latent dims 256-511: A from tensor memory, 8 columns per K = 16 step
+              if (kPhase && st == 2) {  // output-phase: dims 256-319 from shared memory, 320-383 from tensor memory
+                const uint64_t da = umma_desc_sw128(q_base + 4 * kQChunkBytes, 16, 1024), db = umma_desc_sw128(b_addr, 16, 1024);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_f16<2>(tmem_s, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), kIdescQK, 1u);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                  umma_f16_ts<2>(tmem_s, tmem_base + kColQp + 8u * k, db + (uint64_t)((kChunkBytes + k * 32) >> 4), kIdescQK, 1u);
+                umma_commit_2_mc(bar(C::kBarRingEmpty + s), 3);
+              } else if (kPhase && st == 3) {  // output-phase: dims 384-511 from tensor memory
+                const uint64_t db = umma_desc_sw128(b_addr, 16, 1024);
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                  umma_f16_ts<2>(tmem_s, tmem_base + kColQp + 32u + 8u * k,
+                                 db + (uint64_t)(((k >> 2) * kChunkBytes + (k & 3) * 32) >> 4), kIdescQK, 1u);
+                umma_commit_2_mc(bar(C::kBarRingEmpty + s), 3);
+              } else if (!kPhase && st >= 2 && st < 4) {  // latent dims 256-511: A from tensor memory, 8 columns per K = 16 step
                 const uint32_t a_tmem = tmem_base + kColQ + (uint32_t)(st - 2) * 64u;
                 const uint64_t db = umma_desc_sw128(b_addr, 16, 1024);
 #pragma unroll
@@ -469,7 +490,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
                                  kIdescQK, 1u);
                 }
                 umma_commit_2_mc(bar(C::kBarRingEmpty + s), 3);
-              } else if (st < C::kQSmemChunks / 2) {  // latent dims held in shared memory
+              } else if (st < 2) {  // latent dims 0-255: A from shared memory
                 const uint32_t a_addr = q_base + 2 * st * kQChunkBytes;
                 // descriptors differ only in the start-address field (16-byte units): add constants
                 const uint64_t da = umma_desc_sw128(a_addr, 16, 1024), db = umma_desc_sw128(b_addr, 16, 1024);
@@ -576,6 +597,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       const AttnWorkItem item = get_work(p, w);
       ok = mbar_wait_bounded<false>(bar(C::kBarQFull), qfull_phase, limit, abort_flag, p.status, W_QFULL, w);
       qfull_phase ^= 1;
+      uint4 pr[16];  // output-phase: the rope chunk as loaded, this lane's 16 pieces (it landed in a rotated buffer)
+      if constexpr (kPhase) {
+        if (ok) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int idx = lane + 32 * i;
+            pr[i] = *reinterpret_cast<const uint4*>(smem + C::kOffQPristine + sw128_offset((uint32_t)(idx >> 3), (uint32_t)(idx & 7)));
+          }
+        }
+        __syncwarp();  // every lane has its pieces before any lane overwrites the buffer
+      }
       SegIter it(p, item);
       while (ok && it.next()) {
         const uint32_t rb = qr_use & 1u;
@@ -589,12 +621,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         const float2* cs = p.seg_cs + (size_t)it.seg * 32;
         const uint8_t* src = smem + C::kOffQPristine;
         uint8_t* dst = smem + C::kOffQRot + rb * kQChunkBytes;
-#pragma unroll 4
+#pragma unroll(kPhase ? 16 : 4)
         for (int i = 0; i < 16; ++i) {
           const int idx = lane + 32 * i;
           const uint32_t row = idx >> 3, c = idx & 7;
           const uint32_t off = sw128_offset(row, c);
-          uint4 v = *reinterpret_cast<const uint4*>(src + off);
+          uint4 v;
+          if constexpr (kPhase) v = pr[i]; else v = *reinterpret_cast<const uint4*>(src + off);
           uint32_t in[4] = {v.x, v.y, v.z, v.w};
           uint32_t outv[4];
 #pragma unroll
@@ -661,7 +694,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
       }
       float m_run = -INFINITY, l_run = 0.f;
       int kt = 0;
-      if constexpr (!kPhase) {  // move this thread's share of the upper Q half (row m, 64 dims) from its ring stage into TMEM
+      {  // move this thread's share of the upper Q part (row m) from its ring stage into TMEM
         ok = mbar_wait_bounded<false>(bar(C::kBarQhFull), qh_full_phase, limit, abort_flag, p.status, W_QHFULL, w);
         qh_full_phase ^= 1;
         if (!ok) break;
@@ -670,6 +703,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         ring_it += 1u + (uint32_t)C::kStagesPerKeyTile * (uint32_t)count_key_tiles(p, item);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
+          if (2 * ch + half >= C::kQTmemChunks) continue;  // output-phase: three chunks only (warp-uniform)
           uint32_t qv[32];
           const uint8_t* chunk = stage + (2 * ch + half) * kQChunkBytes;
 #pragma unroll
@@ -677,7 +711,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
             const uint4 v = *reinterpret_cast<const uint4*>(chunk + sw128_offset((uint32_t)m, (uint32_t)c));
             qv[4 * c] = v.x; qv[4 * c + 1] = v.y; qv[4 * c + 2] = v.z; qv[4 * c + 3] = v.w;
           }
-          tmem_st_x32(tmem_base + lane_base + kColQ + (uint32_t)(ch * 64 + half * 32), qv);
+          tmem_st_x32(tmem_base + lane_base + (kPhase ? kColQp : kColQ) + (uint32_t)(ch * 64 + half * 32), qv);
         }
         tmem_wait_st();
         tc_fence_before_sync();
