@@ -82,10 +82,13 @@ def test_phase_large_offsets_and_gaps(rk):
     check_every_row(rk, w)
 
 
-@pytest.mark.parametrize("regime", ["mandated", "sharp"])
-def test_phase_full_size_flash1_sampled_rows(rk, regime):
-    prof, lay, prot = synth.make_geometry("flash1")
-    w = synth.make_tensors("flash1", prof, lay, prot, 1000, device="cuda", regime=regime, value_phase=True)
+@pytest.mark.parametrize("name, regime", [("flash1", "mandated"), ("flash1", "sharp"), ("flash256k", "sharp")])
+def test_phase_full_size_sampled_rows(rk, name, regime):
+    """Full-size layers of the variant in the launch configuration `bench.py --value-phase` times (flash256k is its
+    workload); sampled rows against the checker."""
+    prof, lay, prot = synth.make_geometry(name)
+    w = synth.make_tensors(name, prof, lay, prot, synth.CONFIGS[name]["seed"] * 1000, device="cuda", regime=regime,
+                           value_phase=True)
     ctx, req = make(rk, w)
     O_g, lse_g, O_l, lse_l, z, y = layer(ctx, req, w)
     cand = synth.sample_rows(lay, prot, 16, w.seed, max_docs=3)
@@ -94,7 +97,7 @@ def test_phase_full_size_flash1_sampled_rows(rk, regime):
     rows, used = [], 0
     for r in np.random.default_rng(3).permutation(cand):
         c = (int(pos[r]) + 1) * (prof.n_heads if inv[r] >= 0 else prof.n_groups)
-        if used + c > 3e7 and len(rows) >= 4:
+        if used + c > (3e7 if name == "flash1" else 6e7) and len(rows) >= 4:
             continue
         rows.append(int(r))
         used += c
@@ -177,3 +180,31 @@ def test_segmented_merge_phase(rk, dtype):
     assert max_abs(f64(lse)[fin], want_lse[fin]) <= 1e-3
     assert_close(f64(O), want_O, "merged O with part phases and R^-1", unit_scale=True)
     assert_close(f64(O2), want_O2, "merged O in the request frame", unit_scale=True)
+
+
+def test_phase_layer_stack_host_matches_device_path(rk):
+    """Three independent layers of the variant through the stack entry point with cross-layer prefetch:
+    bit-identical to the call-by-call device path."""
+    layers, want = [], []
+    ctx = None
+    for l in range(3):
+        prof, lay, prot = synth.make_geometry("tiny", layer=l)
+        prot = synth.draw_protected_rows(lay, 300 + 300 * l, np.random.default_rng(200 + l))
+        w = synth.make_tensors("tiny", prof, lay, prot, 700 + l, regime="sharp", value_phase=True)
+        if ctx is None:
+            ctx = rk.Context.from_profile(prof, value_phase=True)
+        req = ctx.rk_request_create(lay.seg_off, lay.seg_delta, lay.seg_has_artifact, prot)
+        pin = lambda t: t.cpu().pin_memory()
+        host = dict(req=req, kv=pin(w.kv), q_g=pin(w.q_g), q_l=pin(w.q_l), z_off=pin(w.z_off))
+        to_device(w)
+        _, _, _, _, _, y = layer(ctx, req, w)
+        want.append(y.cpu())
+        host.update(W_uv=w.w_uv, W_a=w.w_a, W_b=w.w_b,
+                    y=torch.full((lay.n_rows, prof.d_model), float("nan"), dtype=torch.bfloat16).pin_memory())
+        layers.append(host)
+    big = max(layers, key=lambda l: l["req"].A)["req"]
+    b0, b1 = ctx.alloc_layer_buffers(big, "cuda"), ctx.alloc_layer_buffers(big, "cuda")
+    rk.rk_layer_stack_host(ctx, layers, b0, b1)
+    ctx.rk_poll_status()
+    for l in range(3):
+        assert torch.equal(layers[l]["y"], want[l]), f"layer {l}"
