@@ -453,7 +453,9 @@ def main():
         for i, (wl, r) in enumerate(layers):
             run_layer(wl, r, ev[i] if ev else None)
 
-    launches_per_step = (2 + 4 + 1 + 1) * n_layers   # per layer: attention x2, projection GEMMs x4, combine, W_b
+    # per layer: attention x2; sliced projection: Global half fused (1 launch) when r_o is a multiple of 256, else 2,
+    # Local half 2; combine; W_b
+    launches_per_step = (2 + (1 if prof.o_rank % 256 == 0 else 2) + 2 + 1 + 1) * n_layers
 
     for _ in range(args.warmup):
         step()

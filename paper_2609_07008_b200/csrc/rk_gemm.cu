@@ -489,3 +489,323 @@ cudaError_t launch_gemm(const GemmParams& p, int bn, int sm_count, cudaStream_t 
 }
 
 }  // namespace rk
+
+// ------------------------------------------------------------------------------------------------------
+// Fused sliced first projection of the Global heads (Eq. offonline): per (128-row block, group g)
+//   o[128 x 128]   = O_g[rows, g] W_uv[head_g]^T            (K = 512, or 576 in the output-phase variant)
+//   z[128 x r_o]   = o W_a[g][:, 128 j_g : 128 j_g + 128]^T  (K = 128), written as r_o / 128 column tiles
+// with o kept on chip: the first accumulator is converted to bf16 into a shared-memory tile that is the A
+// operand of the second contraction, so the 128-wide intermediate never travels to memory and back.  HBM
+// traffic is O_g once in and z_on_g once out.  One CTA per SM, persistent over (row block, group) tiles in that
+// order; warp 0 TMA producer, warp 1 UMMA issuer, warps 4-11 two epilogue groups of four warps.
+// ------------------------------------------------------------------------------------------------------
+namespace rk {
+namespace {
+
+constexpr int kFpThreads = 384;
+constexpr int kFpStages = 4;
+struct FpSmem {
+  static constexpr uint32_t kStageBytes = 32768;                   // GEMM1: A chunk + W_uv chunk; GEMM2: two W_a chunks
+  static constexpr uint32_t kOffO = kFpStages * kStageBytes;       // o tile, bf16 [128 x 128] as two K-major 128B-swizzled chunks
+  static constexpr uint32_t kOffCStage = kOffO + 32768;            // four 16 KB output staging tiles (two per epilogue group)
+  static constexpr uint32_t kOffBars = kOffCStage + 4 * 16384;
+  // full[4], empty[4], acc1_full, acc1_empty, o_ready, o_free, acc2_full[3], acc2_empty[3]
+  static constexpr int kBarFull = 0, kBarEmpty = kFpStages, kBarAcc1Full = 2 * kFpStages, kBarAcc1Empty = kBarAcc1Full + 1,
+                       kBarOReady = kBarAcc1Empty + 1, kBarOFree = kBarOReady + 1, kBarAcc2Full = kBarOFree + 1,
+                       kBarAcc2Empty = kBarAcc2Full + 3, kNumBars = kBarAcc2Empty + 3;
+  static constexpr uint32_t kOffTmemPtr = kOffBars + kNumBars * 8;
+  static constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
+  static constexpr uint32_t kBytes = kOffAbort + 8 + 1024;
+};
+enum { WF_FULL = 41, WF_EMPTY, WF_ACC1_FULL, WF_ACC1_EMPTY, WF_O_READY, WF_O_FREE, WF_ACC2_FULL, WF_ACC2_EMPTY };
+
+__global__ void __launch_bounds__(kFpThreads, 1) rk_proj_fused_kernel(const __grid_constant__ FusedProjParams p) {
+  using S = FpSmem;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  auto bar = [&](int i) -> uint32_t { return smem_base + S::kOffBars + 8u * i; };
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::kOffAbort);
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + S::kOffTmemPtr);
+  const uint64_t limit = p.wait_ns;
+  const int n_mb = (p.M + kBM - 1) / kBM;
+  const int n_tiles = n_mb * p.n_groups;
+  const int k1_chunks = p.K1 / kBK;
+  const int n_nt = p.o_rank / 128;  // column tiles of the second contraction
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < kFpStages; ++s) {
+      mbar_init(bar(S::kBarFull + s), 1);
+      mbar_init(bar(S::kBarEmpty + s), 1);
+    }
+    mbar_init(bar(S::kBarAcc1Full), 1);
+    mbar_init(bar(S::kBarAcc1Empty), 8);  // every epilogue warp has read its part of the first accumulator
+    mbar_init(bar(S::kBarOReady), 8);     // ... and written its part of o
+    mbar_init(bar(S::kBarOFree), 1);      // the second contraction of the tile has finished reading o
+    for (int b = 0; b < 3; ++b) {
+      mbar_init(bar(S::kBarAcc2Full + b), 1);
+      mbar_init(bar(S::kBarAcc2Empty + b), 4);  // the four warps of the group that read it
+    }
+    fence_mbar_init_cluster();
+  }
+  if (warp == 0) {
+    __syncwarp();
+    tmem_alloc<1>(smem_base + S::kOffTmemPtr, 512);
+    tmem_relinquish<1>();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_ptr_smem;
+  // acc2: a ring of three 128-column buffers, so that the MMAs of the next column tiles run while a tile is being
+  // stored (with one buffer per epilogue group the group idled for the whole empty -> MMA -> full round trip of
+  // every column tile: 18.5K instead of about 8K clk per row-block tile)
+  constexpr uint32_t kColAcc1 = 0, kColAcc2 = 128;
+
+  // Order of the ring (producer and issuer walk it alike): the first contraction of the first tile, then for every
+  // tile its second contraction's column tiles interleaved one to one with the k-chunks of the NEXT tile's first
+  // contraction.  So the next tile's o accumulates while this tile's z is being stored, and the store path (the
+  // slowest part: an SM writes about 26 bytes per clock) never waits for a first contraction.
+  if (warp == 0) {
+    // ---- TMA producer ----
+    if (lane == 0) {
+      tma_prefetch_desc(&p.tm_a);
+      tma_prefetch_desc(&p.tm_b1);
+      tma_prefetch_desc(&p.tm_b2);
+    }
+    uint32_t it = 0;
+    bool ok = true;
+    auto acquire = [&](int t) -> bool {
+      const uint32_t s = it % kFpStages;
+      if (it >= (uint32_t)kFpStages)
+        return mbar_wait_bounded<false>(bar(S::kBarEmpty + s), ((it / kFpStages) & 1u) ^ 1u, limit, abort_flag, p.status, WF_EMPTY, t);
+      return true;
+    };
+    auto load1 = [&](int t, int kc) -> bool {  // k-chunk kc of tile t's first contraction: A chunk + W_uv chunk
+      if (!acquire(t)) return false;
+      if (elect_one()) {
+        const int mb = t / p.n_groups, g = t - mb * p.n_groups;
+        const GemmBatch b1 = p.batches_uv[g];
+        const uint32_t s = it % kFpStages, dst = smem_base + s * S::kStageBytes;
+        mbar_arrive_expect_tx(bar(S::kBarFull + s), S::kStageBytes);
+        tma_load_2d(dst, &p.tm_a, bar(S::kBarFull + s), b1.a_col0 + kc * kBK, mb * kBM);
+        tma_load_2d(dst + 16384, &p.tm_b1, bar(S::kBarFull + s), kc * kBK, b1.b_row0);
+      }
+      __syncwarp();
+      ++it;
+      return true;
+    };
+    auto load2 = [&](int t, int nt) -> bool {  // column tile nt of tile t's second contraction: two W_a chunks
+      if (!acquire(t)) return false;
+      if (elect_one()) {
+        const int mb = t / p.n_groups, g = t - mb * p.n_groups;
+        const GemmBatch b2 = p.batches_wa[g];
+        const uint32_t s = it % kFpStages, dst = smem_base + s * S::kStageBytes;
+        mbar_arrive_expect_tx(bar(S::kBarFull + s), S::kStageBytes);
+        tma_load_2d(dst, &p.tm_b2, bar(S::kBarFull + s), b2.b_col0, b2.b_row0 + nt * 128);
+        tma_load_2d(dst + 16384, &p.tm_b2, bar(S::kBarFull + s), b2.b_col0 + kBK, b2.b_row0 + nt * 128);
+      }
+      __syncwarp();
+      ++it;
+      return true;
+    };
+    if ((int)blockIdx.x < n_tiles)
+      for (int kc = 0; kc < k1_chunks && ok; ++kc) ok = load1(blockIdx.x, kc);
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+      const int t_next = t + gridDim.x;
+      const int n1 = t_next < n_tiles ? k1_chunks : 0;
+      for (int j = 0; (j < n_nt || j < n1) && ok; ++j) {
+        if (j < n_nt) ok = load2(t, j);
+        if (ok && j < n1) ok = load1(t_next, j);
+      }
+    }
+    for (uint32_t back = 1; back <= (uint32_t)kFpStages && ok; ++back) {
+      if (it >= back) {
+        const uint32_t u = it - back;
+        ok = mbar_wait_bounded<false>(bar(S::kBarEmpty + u % kFpStages), (u / kFpStages) & 1u, limit, abort_flag, p.status, WF_EMPTY, -1);
+      }
+    }
+  } else if (warp == 1) {
+    // ---- UMMA issuer ----
+    constexpr uint32_t idesc = umma_idesc_bf16(kBM, 128, 0, 0);
+    uint32_t it = 0, tile_i = 0, use2 = 0;  // use2: column tiles issued so far (buffer = use2 % 3)
+    bool ok = true;
+    const uint32_t o_addr = smem_base + S::kOffO;
+    auto mma1 = [&](int t, int kc) -> bool {  // one k-chunk of a first contraction into acc1
+      const uint32_t s = it % kFpStages;
+      if (!mbar_wait_bounded<false>(bar(S::kBarFull + s), (it / kFpStages) & 1u, limit, abort_flag, p.status, WF_FULL, t)) return false;
+      const uint32_t a_addr = smem_base + s * S::kStageBytes;
+      if (elect_one()) {
+        const uint64_t da = umma_desc_sw128(a_addr, 16, 1024), db = umma_desc_sw128(a_addr + 16384, 16, 1024);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_f16<1>(tmem_base + kColAcc1, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kc > 0 || k > 0) ? 1u : 0u);
+        umma_commit_1(bar(S::kBarEmpty + s));
+        if (kc == k1_chunks - 1) umma_commit_1(bar(S::kBarAcc1Full));
+      }
+      __syncwarp();
+      ++it;
+      return true;
+    };
+    auto mma2 = [&](int t, int nt) -> bool {  // one column tile of a second contraction into the next acc2 buffer
+      const uint32_t e = use2 % 3u, u = use2 / 3u;  // u-th use of buffer e
+      if (u >= 1) {
+        if (!mbar_wait_bounded<false>(bar(S::kBarAcc2Empty + e), (u - 1) & 1u, limit, abort_flag, p.status, WF_ACC2_EMPTY, t)) return false;
+        tc_fence_after_sync();
+      }
+      const uint32_t s = it % kFpStages;
+      if (!mbar_wait_bounded<false>(bar(S::kBarFull + s), (it / kFpStages) & 1u, limit, abort_flag, p.status, WF_FULL, t)) return false;
+      const uint32_t b_addr = smem_base + s * S::kStageBytes;
+      if (elect_one()) {
+        const uint64_t da = umma_desc_sw128(o_addr, 16, 1024), db = umma_desc_sw128(b_addr, 16, 1024);
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          umma_f16<1>(tmem_base + kColAcc2 + e * 128u, da + (uint64_t)(((k >> 2) * 16384 + (k & 3) * 32) >> 4),
+                      db + (uint64_t)(((k >> 2) * 16384 + (k & 3) * 32) >> 4), idesc, k > 0 ? 1u : 0u);
+        umma_commit_1(bar(S::kBarEmpty + s));
+        umma_commit_1(bar(S::kBarAcc2Full + e));
+        if (nt == n_nt - 1) umma_commit_1(bar(S::kBarOFree));
+      }
+      __syncwarp();
+      ++it;
+      ++use2;
+      return true;
+    };
+    if ((int)blockIdx.x < n_tiles)
+      for (int kc = 0; kc < k1_chunks && ok; ++kc) ok = mma1(blockIdx.x, kc);
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
+      const int t_next = t + gridDim.x;
+      const int n1 = t_next < n_tiles ? k1_chunks : 0;
+      // o of this tile is in shared memory; that also means the epilogue has read acc1, so the next tile's first
+      // contraction may overwrite it
+      ok = mbar_wait_bounded<false>(bar(S::kBarOReady), tile_i & 1u, limit, abort_flag, p.status, WF_O_READY, t) &&
+           mbar_wait_bounded<false>(bar(S::kBarAcc1Empty), tile_i & 1u, limit, abort_flag, p.status, WF_ACC1_EMPTY, t);
+      if (!ok) break;
+      tc_fence_after_sync();
+      for (int j = 0; (j < n_nt || j < n1) && ok; ++j) {
+        if (j < n_nt) ok = mma2(t, j);
+        if (ok && j < n1) ok = mma1(t_next, j);
+      }
+    }
+  } else if (warp >= 4) {
+    // ---- epilogue: group e owns o chunk e (64 columns of the first accumulator) and every other column tile ----
+    const int e = (warp - 4) >> 2;
+    const int L = (threadIdx.x - 128) & 127;
+    const int bar_id = 1 + e;
+    const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
+    uint32_t tile_i = 0, chunk_i = 0;
+    bool ok = true;
+    if (L == 0) tma_prefetch_desc(&p.tm_c);
+    // o of tile number i (in this CTA's sequence): first accumulator -> bf16 -> shared-memory A tile of the second
+    // contraction.  It runs before the group's last column tile of the previous row-block tile, so that the
+    // second contraction of the next tile is already under way when the stores of this one end.
+    auto convert_o = [&](uint32_t i, int t) -> bool {
+      bool good = mbar_wait_bounded<false>(bar(S::kBarAcc1Full), i & 1u, limit, abort_flag, p.status, WF_ACC1_FULL, t);
+      if (good && i >= 1)
+        good = mbar_wait_bounded<false>(bar(S::kBarOFree), (i - 1) & 1u, limit, abort_flag, p.status, WF_O_FREE, t);
+      good = named_barrier_and(bar_id, 128, good);
+      if (!good) return false;
+      tc_fence_after_sync();
+      uint32_t o[64];
+      tmem_ld_x32(tmem_base + lane_base + kColAcc1 + 64u * e, o);
+      tmem_ld_x32(tmem_base + lane_base + kColAcc1 + 64u * e + 32, o + 32);
+      tmem_wait_ld();
+      tc_fence_before_sync();
+      uint8_t* dst = smem + S::kOffO + e * 16384;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(o[8 * c + 0]), __uint_as_float(o[8 * c + 1]));
+        v.y = pack_bf16(__uint_as_float(o[8 * c + 2]), __uint_as_float(o[8 * c + 3]));
+        v.z = pack_bf16(__uint_as_float(o[8 * c + 4]), __uint_as_float(o[8 * c + 5]));
+        v.w = pack_bf16(__uint_as_float(o[8 * c + 6]), __uint_as_float(o[8 * c + 7]));
+        *reinterpret_cast<uint4*>(dst + sw128_offset((uint32_t)L, (uint32_t)c)) = v;
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(bar(S::kBarAcc1Empty));
+        mbar_arrive(bar(S::kBarOReady));
+      }
+      return true;
+    };
+    if ((int)blockIdx.x < n_tiles) ok = convert_o(0, blockIdx.x);
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
+      const int mb = t / p.n_groups, g = t - mb * p.n_groups;
+      const GemmBatch b2 = p.batches_wa[g];
+      const int m0 = mb * kBM;
+      const int t_next = t + gridDim.x;
+      // ---- z: this group's column tiles ----
+      for (int nt = e; nt < n_nt && ok; nt += 2) {
+        if (nt + 2 >= n_nt && t_next < n_tiles) {  // before this group's last column tile: the next tile's o
+          ok = convert_o(tile_i + 1, t_next);
+          if (!ok) break;
+        }
+        const uint32_t q = tile_i * (uint32_t)n_nt + (uint32_t)nt;  // column tiles are issued in this order
+        const uint32_t b = q % 3u, u = q / 3u;
+        ok = mbar_wait_bounded<false>(bar(S::kBarAcc2Full + b), u & 1u, limit, abort_flag, p.status, WF_ACC2_FULL, t);
+        ok = named_barrier_and(bar_id, 128, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+#pragma unroll 1
+        for (int cc = 0; cc < 128; cc += 64, ++chunk_i) {
+          uint32_t o[64];
+          tmem_ld_x32(tmem_base + lane_base + kColAcc2 + 128u * b + cc, o);
+          tmem_ld_x32(tmem_base + lane_base + kColAcc2 + 128u * b + cc + 32, o + 32);
+          tmem_wait_ld();
+          if (cc == 64) {
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(S::kBarAcc2Empty + b));
+          }
+          const uint32_t buf = 2u * e + (chunk_i & 1u);
+          if (L == 0) bulk_wait_group_read<1>();
+          named_barrier_sync(bar_id, 128);
+          uint8_t* stage = smem + S::kOffCStage + buf * 16384;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(o[8 * c + 0]), __uint_as_float(o[8 * c + 1]));
+            v.y = pack_bf16(__uint_as_float(o[8 * c + 2]), __uint_as_float(o[8 * c + 3]));
+            v.z = pack_bf16(__uint_as_float(o[8 * c + 4]), __uint_as_float(o[8 * c + 5]));
+            v.w = pack_bf16(__uint_as_float(o[8 * c + 6]), __uint_as_float(o[8 * c + 7]));
+            *reinterpret_cast<uint4*>(stage + sw128_offset((uint32_t)L, (uint32_t)c)) = v;
+          }
+          fence_proxy_async_smem();
+          named_barrier_sync(bar_id, 128);
+          if (L == 0) {
+            tma_store_2d(&p.tm_c, smem_base + S::kOffCStage + buf * 16384, b2.c_col0 + nt * 128 + cc, m0);
+            bulk_commit_group();
+          }
+        }
+      }
+    }
+    if (L == 0) bulk_wait_group<0>();
+  }
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    __syncwarp();
+    tmem_dealloc<1>(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+cudaError_t proj_fused_setup() {
+  return cudaFuncSetAttribute(rk_proj_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FpSmem::kBytes);
+}
+
+cudaError_t launch_proj_fused(const FusedProjParams& p, int sm_count, cudaStream_t stream) {
+  const long long tiles = (long long)((p.M + kBM - 1) / kBM) * p.n_groups;
+  if (tiles <= 0) return cudaSuccess;
+  const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+  rk_proj_fused_kernel<<<grid, kFpThreads, FpSmem::kBytes, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace rk

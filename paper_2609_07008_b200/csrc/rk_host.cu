@@ -270,6 +270,7 @@ rk_status rk_create_ex(const rk_profile* prof, uint32_t flags, rk_ctx** out) {
   e = attention_setup();
   if (e == cudaSuccess) e = gemm_setup();
   if (e == cudaSuccess) e = stream_setup();
+  if (e == cudaSuccess) e = proj_fused_setup();
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->d_status), sizeof(DeviceStatus));
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(DeviceStatus));
   if (e != cudaSuccess) {
@@ -779,6 +780,39 @@ static rk_status run_gemm(rk_ctx* ctx, const void* A, int64_t a_rows, int64_t a_
   return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "gemm launch");
 }
 
+// Global half of the sliced first projection for `n` rows: one fused kernel when the group rank is a multiple of
+// 256 (o = W_uv O stays on chip), else the two batched GEMMs with o in the workspace.
+static rk_status proj_global(rk_ctx* ctx, const void* O_g, int64_t n, const void* W_uv, const void* W_a, void* o_g,
+                             void* z_on_g, cudaStream_t st) {
+  const int G = ctx->prof.n_groups, H = ctx->prof.n_heads, ro = ctx->prof.o_rank;
+  if (n == 0) return RK_OK;
+  if (ro % 256 == 0) {
+    FusedProjParams p;
+    memset(&p, 0, sizeof(p));
+    rk_status s = make_tmap(ctx, &p.tm_a, O_g, (uint64_t)n, (uint64_t)G * ctx->ow, (uint64_t)G * ctx->ow, 64, 128);
+    if (s == RK_OK) s = make_tmap(ctx, &p.tm_b1, W_uv, (uint64_t)H * kDV, (uint64_t)ctx->ow, (uint64_t)ctx->ow, 64, 128);
+    if (s == RK_OK) s = make_tmap(ctx, &p.tm_b2, W_a, (uint64_t)G * ro, (uint64_t)kGroup * kDV, (uint64_t)kGroup * kDV, 64, 128);
+    if (s == RK_OK) s = make_tmap(ctx, &p.tm_c, z_on_g, (uint64_t)n, (uint64_t)G * ro, (uint64_t)G * ro, 64, 128);
+    if (s != RK_OK) return s;
+    p.batches_uv = ctx->d_batches + ctx->off_uv_g;
+    p.batches_wa = ctx->d_batches + ctx->off_wa_g;
+    p.status = ctx->d_status;
+    p.wait_ns = ctx->wait_ns;
+    p.M = (int32_t)n;
+    p.n_groups = G;
+    p.K1 = ctx->ow;
+    p.o_rank = ro;
+    cudaError_t e = launch_proj_fused(p, ctx->sm_count, st);
+    return e == cudaSuccess ? RK_OK : cuda_fail(ctx, e, "fused projection launch");
+  }
+  rk_status s = run_gemm(ctx, O_g, n, (int64_t)G * ctx->ow, W_uv, (int64_t)H * kDV, ctx->ow, o_g, (int64_t)G * kDV, (int)n, kDV,
+                         ctx->ow, ctx->off_uv_g, G, st);
+  if (s == RK_OK)
+    s = run_gemm(ctx, o_g, n, (int64_t)G * kDV, W_a, (int64_t)G * ro, kGroup * kDV, z_on_g, (int64_t)G * ro, (int)n, ro, kDV,
+                 ctx->off_wa_g, G, st);
+  return s;
+}
+
 rk_status rk_group_sliced_proj(rk_ctx* ctx, const rk_request* rq, const void* O_g, const void* O_l, const void* W_uv,
                                const void* W_a, void* z_on_g, void* z_on_l, void* workspace, size_t workspace_bytes,
                                void* stream) {
@@ -799,13 +833,7 @@ rk_status rk_group_sliced_proj(rk_ctx* ctx, const rk_request* rq, const void* O_
   void* o_g = ws;
   void* o_l = ws + (((size_t)T * G * kDV * 2 + 255) & ~(size_t)255);
   rk_status s = RK_OK;
-  if (do_g) {
-    s = run_gemm(ctx, O_g, T, (int64_t)G * ctx->ow, W_uv, (int64_t)H * kDV, ctx->ow, o_g, (int64_t)G * kDV, (int)T, kDV,
-                 ctx->ow, ctx->off_uv_g, G, st);
-    if (s == RK_OK)
-      s = run_gemm(ctx, o_g, T, (int64_t)G * kDV, W_a, (int64_t)G * ro, kGroup * kDV, z_on_g, (int64_t)G * ro, (int)T, ro,
-                   kDV, ctx->off_wa_g, G, st);
-  }
+  if (do_g) s = proj_global(ctx, O_g, T, W_uv, W_a, o_g, z_on_g, st);
   if (s == RK_OK && do_l && A > 0) {
     s = run_gemm(ctx, O_l, A, (int64_t)L * ctx->ow, W_uv, (int64_t)H * kDV, ctx->ow, o_l, (int64_t)L * kDV, (int)A, kDV,
                  ctx->ow, ctx->off_uv_l, L, st);
@@ -890,11 +918,8 @@ static rk_status layer_compute(rk_ctx* ctx, const rk_request* rq, const rk_layer
     s = attn_pass(ctx, rq, dev->kv, dev->q_g, T, G, nullptr, n_chunks == 2 ? rq->d_work_g_part[c] : rq->d_work_g,
                   n_chunks == 2 ? rq->n_tiles_g_part[c] : rq->n_tiles_g, dev->O_g, dev->lse_g, st);
     if (s == RK_OK)
-      s = run_gemm(ctx, Og + (size_t)r0 * G * ctx->ow * 2, n, (int64_t)G * ctx->ow, W_uv, (int64_t)H * kDV, ctx->ow,
-                   og + (size_t)r0 * G * kDV * 2, (int64_t)G * kDV, (int)n, kDV, ctx->ow, ctx->off_uv_g, G, st);
-    if (s == RK_OK)
-      s = run_gemm(ctx, og + (size_t)r0 * G * kDV * 2, n, (int64_t)G * kDV, W_a, (int64_t)G * ro, kGroup * kDV,
-                   zg + (size_t)r0 * width * 2, (int64_t)G * ro, (int)n, ro, kDV, ctx->off_wa_g, G, st);
+      s = proj_global(ctx, Og + (size_t)r0 * G * ctx->ow * 2, n, W_uv, W_a, og + (size_t)r0 * G * kDV * 2,
+                      zg + (size_t)r0 * width * 2, st);
     if (s != RK_OK) return s;
     if (c == 0) {  // the artifact has to be there from here on
       e = cudaStreamWaitEvent(st, ev_zoff, 0);

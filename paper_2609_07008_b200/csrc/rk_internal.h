@@ -81,6 +81,21 @@ cudaError_t gemm_setup();
 // single-batch launches with N a multiple of 256 run on CTA pairs; their B tensor map needs a 128-row box
 bool gemm_uses_pairs(int M, int N, int n_batches);
 
+// fused sliced first projection of the Global heads: o = O_g W_uv^T stays on chip, z_on_g = o W_a[slice]^T
+struct FusedProjParams {
+  CUtensorMap tm_a;   // O_g  [M][G * ow]      box 64 x 128
+  CUtensorMap tm_b1;  // W_uv [H * 128][ow]    box 64 x 128
+  CUtensorMap tm_b2;  // W_a  [G * r_o][1024]  box 64 x 128
+  CUtensorMap tm_c;   // z_on_g [M][G * r_o]   box 64 x 128 (stores)
+  const GemmBatch* batches_uv;  // per group: a_col0 = g * ow, b_row0 = Global head * 128
+  const GemmBatch* batches_wa;  // per group: b_row0 = g * r_o, b_col0 = 128 * slot of the Global head, c_col0 = g * r_o
+  DeviceStatus* status;
+  unsigned long long wait_ns;
+  int32_t M, n_groups, K1, o_rank;
+};
+cudaError_t launch_proj_fused(const FusedProjParams& p, int sm_count, cudaStream_t stream);
+cudaError_t proj_fused_setup();
+
 // ---- streaming kernels -----------------------------------------------------------------------
 constexpr int kMergeMaxParts = 4096;  // the merge keeps 8 warps x n_parts weights in shared memory (128 KB at most)
 cudaError_t stream_setup();          // raises the merge kernels' dynamic shared memory limit once
