@@ -39,10 +39,10 @@ FLOP_PER_PAIR = 2 * 576 + 2 * 512     # QK^T over 576 + PV over 512 per visible 
 PROFILED_DRAM_TRAFFIC = {
     "flash256k": dict(bytes=37.41e9 + 9.24e9, algorithmic=4.91e9 + 1.20e9,
                       source="profiles/attn_kernel_flash256k_dram_traffic.md",
-                      captured_on="rk_mla_attn_kernel<kPhase=0, kStarve=0> (template instantiations, no run-time switches)"),
+                      captured_on="commit 4117a6a: rk_mla_attn_kernel<kPhase=0, kStarve=0> (unchanged since for this instantiation)"),
     "flash1": dict(bytes=(352.5e6 + 224.8e6) + (169.3e6 + 74.4e6), algorithmic=(350.3e6 + 277.9e6) + (168.4e6 + 115.5e6),
                    source="profiles/attn_kernel_flash1_ncu_full.md",
-                   captured_on="rk_mla_attn_kernel<kPhase=0, kStarve=0> (template instantiations, no run-time switches)"),
+                   captured_on="commit 4117a6a: rk_mla_attn_kernel<kPhase=0, kStarve=0> (unchanged since for this instantiation)"),
 }
 L2_BYTES = 126 * 1024 * 1024
 
