@@ -350,17 +350,10 @@ def time_offline_build(ctx, req, w, prof, lay, dev, rows_per_call=65536):
             hi = min(n, lo + rows_per_call)
             ctx.rk_mla_off_build(req, w.kv, lo, hi, q[: hi - lo], w.w_uv, w.w_a, z[: hi - lo], ws)
 
-    run()
-    run()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    run()
-    b.record(stream)
-    torch.cuda.synchronize()
+    ms, mhz, mx = timed_region(run, stream, dev.index or 0, min_ms=300.0, lead_ms=50.0)   # steady state, like the other kernels
     ctx.rk_poll_status()
-    ms = a.elapsed_time(b)
     return dict(ms=ms, rows=n, tokens_per_s=n / ms * 1e3, tflops=flops / ms / 1e9, rows_per_call=rows_per_call,
-                flops=flops)
+                flops=flops, sm_mhz=mhz)
 
 
 def main():

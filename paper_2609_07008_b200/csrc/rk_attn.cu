@@ -366,6 +366,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
         for (int d = 0; d < C::kQSmemChunks; ++d)
           tma_load_2d_hint(smem_base + C::kOffQLat + d * kQChunkBytes, &p.tm_q, bar(C::kBarQFull), d * 64, qrow, pol_q);
         tma_load_2d_hint(smem_base + C::kOffQPristine, &p.tm_q, bar(C::kBarQFull), kDLatent, qrow, pol_q);
+        // The next row tile's queries can only be loaded once this tile's QK^T products are done (one Q buffer);
+        // asking for them now puts them into L2, so that load pays the L2 latency instead of the DRAM one.  It
+        // matters where a row tile sees few key tiles (documents built alone: 16 at most).
+        if (w + p.n_pairs < p.n_tiles) {
+          const int qnext = get_work(p, w + p.n_pairs).tile * kAttnRowsPerPair + (int)crank * kAttnRowsPerCta;
+#pragma unroll
+          for (int d = 0; d < 9; ++d) tma_prefetch_2d(&p.tm_q, d * 64, qnext);
+        }
       }
       __syncwarp();
       // Upper latent part (dims 256-511, or 320-511): staged through one ring stage, from where the softmax
