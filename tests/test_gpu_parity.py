@@ -161,6 +161,35 @@ def test_group_sliced_proj(rk):
     assert_close(f64(z2), want2.reshape(A, -1), "z_on_l with one slice zeroed", unit_scale=w.regime == "sharp")
 
 
+@pytest.mark.parametrize("H, G, ro, lens, nq", [
+    (16, 2, 512, [513, 255, 64], 128),     # fused Global kernel, four column tiles
+    (32, 4, 1024, [130, 77], 31),          # eight column tiles, ragged last row block
+    (16, 2, 768, [1000], 5),               # six column tiles
+    (8, 1, 256, [64], 64),                 # one group, exactly one row block
+    (16, 2, 128, [300, 200], 40),          # r_o not a multiple of 256: the two-GEMM path
+])
+def test_group_sliced_proj_shapes(rk, H, G, ro, lens, nq):
+    """The sliced first projection over group ranks and row counts that take every path of its kernels (the Global
+    half is one fused kernel when r_o is a multiple of 256), each against the checker."""
+    w = synth.make_custom(lens, nq, n_heads=H, n_groups=G, o_rank=ro, d_model=256, pct_bp=1500, seed=90 + ro // 128)
+    ctx, req = make(rk, w)
+    p, T, A = w.profile, w.layout.n_rows, len(w.prot_rows)
+    g = torch.Generator().manual_seed(ro)
+    O_g = (torch.randn((T, G, 512), generator=g) * 0.5).to(torch.bfloat16)
+    O_l = (torch.randn((A, H - G, 512), generator=g) * 0.5).to(torch.bfloat16)
+    to_device(w)
+    z_on_g, z_on_l = ctx.rk_group_sliced_proj(req, O_g.cuda(), O_l.cuda(), w.w_uv, w.w_a)
+    ctx.rk_poll_status()
+    wuv, wa = f64(w.w_uv), f64(w.w_a)
+    want_g = oracle.head_contributions(f64(O_g), p.global_heads, wuv, wa).reshape(T, -1)
+    cl = oracle.head_contributions(f64(O_l), p.local_heads, wuv, wa)
+    want_l = np.zeros((A, G, ro))
+    for a, h in enumerate(p.local_heads):
+        want_l[:, h // 8] += cl[:, a]
+    assert_close(f64(z_on_g), want_g, "z_on_g", unit_scale=True)
+    assert_close(f64(z_on_l), want_l.reshape(A, -1), "z_on_l", unit_scale=True)
+
+
 # -- (5) combine + W_b -----------------------------------------------------------------------------------
 
 def test_combine_offline(rk):
