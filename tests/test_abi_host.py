@@ -97,3 +97,15 @@ def test_create_null(rk):
     assert rk.lib.rk_destroy(None) == 1
     assert rk.lib.rk_request_destroy(None) == 1
     assert rk.lib.rk_last_error(None) == b"null context"
+
+
+def test_create_ex_rejects_unknown_flags_and_null_calls_of_the_variant(rk):
+    p, keep = profile_struct(rk)
+    h = C.c_void_p()
+    assert rk.lib.rk_create_ex(C.byref(p), 2, C.byref(h)) == 7          # only RK_VALUE_PHASE (1) is defined
+    assert rk.lib.rk_create_ex(C.byref(p), 0xFFFFFFFE, C.byref(h)) == 7
+    assert not h.value
+    assert rk.lib.rk_create_ex(None, 1, C.byref(h)) == 1
+    assert rk.lib.rk_segmented_merge_phase(None, None, 0, 1, 1, 1, None, 0, None, None, None, None, None) == 1
+    assert rk.lib.rk_check_selftest(None, None) == 1
+    assert rk.lib.rk_test_starve_loads(None, 1) == 1

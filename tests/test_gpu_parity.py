@@ -416,6 +416,14 @@ def test_argument_errors_on_device(rk):
     # merge: unknown part dtype
     assert L.rk_segmented_merge(ctx.handle, 2, 4, 2, O_g.data_ptr(), 7, lse_g.data_ptr(), O_g.data_ptr(),
                                 lse_g.data_ptr(), s) == 7
+    # merge with part phases: segment range beyond the request, too many parts, unknown dtype
+    S = w.layout.n_segs
+    assert L.rk_segmented_merge_phase(ctx.handle, req.handle, 1, S, 4, 2, O_g.data_ptr(), 0, lse_g.data_ptr(), None,
+                                      O_g.data_ptr(), lse_g.data_ptr(), s) == 3
+    assert L.rk_segmented_merge_phase(ctx.handle, req.handle, 0, 4097, 4, 2, O_g.data_ptr(), 0, lse_g.data_ptr(), None,
+                                      O_g.data_ptr(), lse_g.data_ptr(), s) == 3
+    assert L.rk_segmented_merge_phase(ctx.handle, req.handle, 0, 1, 4, 2, O_g.data_ptr(), 5, lse_g.data_ptr(), None,
+                                      O_g.data_ptr(), lse_g.data_ptr(), s) == 7
     # combine: W_b given without y
     assert L.rk_combine_offline(ctx.handle, req.handle, z.data_ptr(), z.data_ptr(), z.data_ptr(), w.w_b.data_ptr(),
                                 z.data_ptr(), None, s) == 1
