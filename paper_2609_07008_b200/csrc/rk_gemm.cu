@@ -561,8 +561,7 @@ __global__ void __launch_bounds__(kFpThreads, 1) rk_proj_fused_kernel(const __gr
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_ptr_smem;
   // acc2: a ring of three 128-column buffers, so that the MMAs of the next column tiles run while a tile is being
-  // stored (with one buffer per epilogue group the group idled for the whole empty -> MMA -> full round trip of
-  // every column tile: 18.5K instead of about 8K clk per row-block tile)
+  // stored (the issuer is up to three column tiles ahead of the epilogue)
   constexpr uint32_t kColAcc1 = 0, kColAcc2 = 128;
 
   // Order of the ring (producer and issuer walk it alike): the first contraction of the first tile, then for every
