@@ -44,6 +44,13 @@ PROFILED_DRAM_TRAFFIC = {
                    source="profiles/attn_kernel_flash1_ncu_full.md",
                    captured_on="commit 4117a6a: rk_mla_attn_kernel<kPhase=0, kStarve=0> (unchanged since for this instantiation)"),
 }
+# Tensor-pipe use counted in SM cycles, from the one-pass ncu capture of the SM clock during the two attention launches
+# (profiles/attn_kernel_flash256k_sm_clock.md): rate / (148 SMs x 8192 flop per clock x measured clock).  A capture's
+# figure, like the traffic above; the NVML clock samples the bench takes itself overstate the clock the kernels get.
+PROFILED_PIPE_USE = {
+    "flash256k": dict(global_pass=0.935, local_pass=0.949, sm_ghz_global=1.317, sm_ghz_local=1.381,
+                      source="profiles/attn_kernel_flash256k_sm_clock.md"),
+}
 L2_BYTES = 126 * 1024 * 1024
 
 
@@ -568,6 +575,7 @@ def main():
                     traffic=None if args.value_phase else (PROFILED_DRAM_TRAFFIC.get(name) or {}).get("bytes"),
                     traffic_note=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("source", "no ncu capture of this workload"),
                     traffic_captured_on=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("captured_on"),
+                    tensor_pipe_use_in_cycles=None if args.value_phase else PROFILED_PIPE_USE.get(name),
                     algorithmic_dram_bytes=(PROFILED_DRAM_TRAFFIC.get(name) or {}).get("algorithmic"))
     rest_tflops = (fl_proj + fl_wb) / (np.mean(rest_ms) * 1e-3) / 1e12
 
