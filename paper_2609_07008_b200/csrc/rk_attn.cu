@@ -25,6 +25,12 @@
 // warp 2 query relocation, warps 4-11 softmax / correction / epilogue (two warps per TMEM lane
 // quarter, each owning half of the columns).  At the start of a row tile the upper Q half lands
 // in one ring stage and the softmax warps copy it into TMEM (tcgen05.st) before their first scores.
+//
+// The kernel is a template: <kPhase = 0> is what the lines above describe.  <kPhase = 1> is the
+// output-phase variant, whose value is the whole stored row (latent and rope dims): a second small
+// accumulator for the 64 rope dims of O, turned into the next segment's frame at every segment
+// switch (RestorePhase of Algorithm 2 folded into the running merge) and by R(delta - pos) in the
+// epilogue (the inverse output RoPE of Eq. offonline); see Cfg for how it fits.
 #include <cuda_bf16.h>
 
 #include "rk_internal.h"

@@ -5,9 +5,14 @@
 // memory -> tcgen05.mma (cta_group::1, M=128, N=BN, K=16) into one of two TMEM accumulators ->
 // tcgen05.ld epilogue that overlaps the next tile's main loop.
 //
-// A batch (blockIdx.z) selects column/row blocks of the 2-D operands: a head's or a group's
-// block.  `b_skip` opens a 128-column hole in B's K axis so that the seven Local slices of a
-// group's W_a are contracted in one pass while the Global head's slice is skipped.
+// A batch selects column/row blocks of the 2-D operands: a head's or a group's block.  `b_skip`
+// opens a 128-column hole in B's K axis so that the seven Local slices of a group's W_a are
+// contracted in one pass while the Global head's slice is skipped.
+//
+// Three kernels live here: rk_gemm_kernel (this general batched form: the Local half of the
+// sliced projection, the offline build, small problems), rk_gemm_pair_kernel (W_b on CTA pairs,
+// cta_group::2 with M = 256) and rk_proj_fused_kernel (the Global half of the sliced projection,
+// both contractions in one kernel with the 128-wide intermediate kept in shared memory).
 #include <cuda_bf16.h>
 
 #include "rk_internal.h"
