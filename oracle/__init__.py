@@ -14,9 +14,10 @@ zero-query and one-hot closed forms, packed-order permutation invariance, global
 invariance, the printed profile ceilings, and torch's scaled_dot_product_attention in
 float64 as a library special case.
 
-parity unpinned: `reuse_error_report` (how far MLA-Online with honest position-zero
-artifacts is from full recomputation on random data) -- the paper quantifies that only
-through model-level F1/EM, so there is nothing to pin it to.
+`reuse_error_report` (how far MLA-Online with honest position-zero artifacts is from full
+recomputation) is pinned as arithmetic by a closed form; the quantity itself, on random data, has
+no value to compare with -- the paper quantifies reuse quality only through model-level F1/EM --
+and no parity claim rests on it.
 """
 from .mla_online import *  # noqa: F401,F403
 from . import phase  # noqa: F401  (output-phase variant: RestorePhase / R^{-1}; pins in tests/test_oracle_phase_pins.py)

@@ -319,8 +319,10 @@ def cold_speed_ratio(s_hot: float, build_units: float = 0.75) -> float:
 
 
 def reuse_error_report(y_online: np.ndarray, y_full: np.ndarray, is_prot: np.ndarray) -> dict:
-    """parity unpinned: relative L2 distance between MLA-Online and full recomputation,
-    split by protected / unprotected rows (a report, not a check)."""
+    """Relative L2 distance between MLA-Online and full recomputation, split by protected /
+    unprotected rows (a report, not a check).  The arithmetic is pinned by a closed form on hand-made
+    vectors; the quantity it reports on random data has no counterpart in the paper (which measures
+    reuse quality through model-level F1 / EM only), so no expected value exists for it."""
     def rel(a, b):
         d = np.linalg.norm(b)
         return float(np.linalg.norm(a - b) / d) if d > 0 else 0.0

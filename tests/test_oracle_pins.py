@@ -397,3 +397,18 @@ def test_wrong_slice_detector():
     d = (z0 - z1).reshape(p["T"], p["G"], p["r_o"])
     assert np.allclose(d[:, g], c, atol=1e-12)
     assert np.allclose(np.delete(d, g, axis=1), 0, atol=1e-13)
+
+
+def test_reuse_error_report_closed_form():
+    """The report is a relative L2 distance on two row subsets: hand-made vectors with known norms."""
+    y_full = np.array([[3.0, 4.0], [0.0, 5.0], [6.0, 8.0], [1.0, 0.0]])          # row norms 5, 5, 10, 1
+    y_on = y_full.copy()
+    y_on[1] += [3.0, 4.0]                                                         # unprotected row off by norm 5
+    y_on[2] += [0.0, 1.0]                                                         # protected row off by norm 1
+    is_prot = np.array([True, False, True, False])
+    rep = oracle.reuse_error_report(y_on, y_full, is_prot)
+    assert abs(rep["protected"] - 1.0 / math.sqrt(25.0 + 100.0)) < 1e-15          # ||(0,0),(0,1)|| / ||rows 0, 2||
+    assert abs(rep["unprotected"] - 5.0 / math.sqrt(25.0 + 1.0)) < 1e-15          # ||(3,4),(0,0)|| / ||rows 1, 3||
+    assert oracle.reuse_error_report(y_full, y_full, is_prot) == dict(protected=0.0, unprotected=0.0)
+    none = oracle.reuse_error_report(y_on, y_full, np.zeros(4, bool))
+    assert none["protected"] == 0.0 and none["unprotected"] > 0
